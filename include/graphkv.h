@@ -1,0 +1,129 @@
+/*
+ * graphkv.h -- C ABI of the GraphKV prefill KV-cache compression library (CUDA, sm_100a).
+ *
+ * GraphKV (paper, Methodology) treats the n prompt tokens of one attention head as graph nodes
+ * o_j with importance scores s_j, takes the top-k nodes as sources (Eq. 2), links each source
+ * to every node by the cosine similarity of their keys (Eq. 1, Algorithm 1), decays the scores
+ * of each source's m most similar neighbours for T rounds (Eq. 3-5, Algorithm 2) and keeps the
+ * k_l highest-scoring tokens' K/V (Problem Formulation: K_s^l, V_s^l).  This library runs that
+ * path at prefill time for all KV heads of a layer on one GPU, with SnapKV-style
+ * observation-window attention as the initial score.
+ *
+ * Conventions common to every call
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library allocates and
+ *     frees nothing; scratch comes from a caller-supplied workspace of at least
+ *     graphkv_workspace_bytes(params) bytes, 256-byte aligned.
+ *   - Calls validate their arguments on the host, enqueue kernels on `stream` (a cudaStream_t
+ *     passed as void*; NULL = the legacy default stream) and return without synchronising.
+ *     The return value reports host-side validation and launch errors only.
+ *   - Layout: Qw [batch][n_q_heads][W][D], K and V [batch][n_kv_heads][L][D] with element
+ *     strides given in the params (D contiguous, every row 16-byte aligned); L = N + W, rows
+ *     [0,N) are the prefix tokens (the graph's nodes), rows [N,L) the observation window.
+ *     KV head h serves query heads [h*G, (h+1)*G), G = n_q_heads / n_kv_heads.
+ *     Outputs are dense: scores [batch][n_kv_heads][N] fp32, idx [batch][n_kv_heads][B] int32,
+ *     K_out / V_out [batch][n_kv_heads][B+W][D] in the input dtype.
+ *   - Every top-k keeps exactly k items; equal values are ordered lower index first, so results
+ *     are deterministic.
+ *   - One workspace serves one call at a time: calls sharing a workspace must be ordered on
+ *     one stream.
+ */
+#ifndef GRAPHKV_H_
+#define GRAPHKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GRAPHKV_OK = 0,
+    GRAPHKV_ERR_INVALID_ARG = 1,   /* NULL pointer, size or stride out of range, misalignment   */
+    GRAPHKV_ERR_UNSUPPORTED = 2,   /* valid but not implemented (head_dim != 128, G*W > 256, ...) */
+    GRAPHKV_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small                 */
+    GRAPHKV_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                          */
+    GRAPHKV_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out (read_status only)      */
+} graphkv_status;
+
+typedef enum { GRAPHKV_BF16 = 0, GRAPHKV_F32 = 1 } graphkv_dtype;
+typedef enum { GRAPHKV_POOL_MAX = 0 } graphkv_pool;
+
+typedef struct {
+    int32_t batch;        /* independent sequences (or any independent units sharing the shape)  */
+    int32_t n_q_heads;
+    int32_t n_kv_heads;   /* must divide n_q_heads                                               */
+    int32_t head_dim;     /* D; 128 required                                                     */
+    int32_t seq_len;      /* L = N + W rows present in K and V                                   */
+    int32_t window;       /* W >= 1 observation-window rows: queried from, always kept           */
+    int32_t budget;       /* B = k_l: prefix tokens kept, 1 <= B <= N; outputs hold B + W rows   */
+    int32_t pool_kernel;  /* odd >= 1 (1 = no pooling); 1-D max pooling of the initial score     */
+    int32_t pool_mode;    /* graphkv_pool                                                        */
+    int32_t topk_nodes;   /* k of Eq. 2: number of source nodes, 0 <= k <= N (0: no propagation) */
+    int32_t neighbors;    /* m of Eq. 3; 0 = adaptive: clamp(floor(N/1000), 1, 32), at most N-1  */
+    int32_t rounds;       /* T of Eq. 5, >= 0; 0 = the base method's plain top-B                 */
+    float   decay;        /* lambda in [0,1], the strength in Eq. 4: factor (1 - lambda*e_ij)    */
+    int32_t dtype;        /* graphkv_dtype of Qw, K, V, K_out, V_out                             */
+    int64_t q_stride[3];  /* element strides of Qw: batch, head, row                             */
+    int64_t k_stride[3];  /* element strides of K: batch, head, token                            */
+    int64_t v_stride[3];  /* element strides of V: batch, head, token                            */
+} graphkv_params;
+
+/* Bytes of scratch any of the calls below needs for these params; 0 if the params are invalid
+ * or unsupported.  Pure host function. */
+size_t graphkv_workspace_bytes(const graphkv_params *params);
+
+/* The neighbour count m the library uses for a prefix of n_prefix tokens when
+ * params.neighbors = `neighbors` (the paper's "Effect of Adjacent Nodes": the smaller of a
+ * preset value and a length-derived one; the length rule is input length x 1e-3). */
+int32_t graphkv_resolve_neighbors(int32_t n_prefix, int32_t neighbors);
+
+/* Step (I) of the pipeline figure, "Initiate Importance Score", with the SnapKV-style score the
+ * paper's Sparse Graph Building section names as one admissible initialisation:
+ *   logits q.k/sqrt(D) of the G*W window rows of each KV head against the prefix keys and the
+ *   causally visible window keys; row softmax; sum over rows and grouped heads of the prefix
+ *   columns; max pooling with pool_kernel.
+ * Reads Qw, K.  Writes scores [batch][n_kv_heads][N] fp32.  Uses topk/decay fields: none. */
+graphkv_status graphkv_score(const graphkv_params *params, const void *Qw, const void *K,
+                             float *scores, void *workspace, size_t workspace_bytes,
+                             void *stream);
+
+/* Steps (II)+(III), "Build Graph" and "Decay Signal Propagation" (Eq. 1-5, Algorithms 1-2):
+ * sources = top-k of `scores`; e_ij = cosine(k_i, k_j) for each source i and every prefix j != i;
+ * N(o_i) = the m largest e_ij; then T times s_j <- s_j * prod_{i: j in N(o_i)} (1 - lambda*max(e_ij,0)).
+ * The graph is built once from the incoming scores and reused by all rounds.
+ * `scores` is updated in place.  src_idx_out (optional, [batch][n_kv_heads][k] int32) receives
+ * the source nodes in ascending position.  With topk_nodes = 0, rounds = 0 or N = 1 the scores
+ * are left unchanged. */
+graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, float *scores,
+                                 int32_t *src_idx_out, void *workspace, size_t workspace_bytes,
+                                 void *stream);
+
+/* Step (IV), "Select Important Tokens": per head the B highest scores (ties: lower index),
+ * written to idx_out in ascending position, and the compact cache
+ *   K_out[b][h][0:B] = K[b][h][idx], K_out[b][h][B:B+W] = K[b][h][N:L]   (same for V),
+ * copied bit for bit.  K/K_out or V/V_out may be NULL together to skip that tensor;
+ * idx_out is required. */
+graphkv_status graphkv_select_gather(const graphkv_params *params, const float *scores,
+                                     const void *K, const void *V, void *K_out, void *V_out,
+                                     int32_t *idx_out, void *workspace, size_t workspace_bytes,
+                                     void *stream);
+
+/* The whole path (I)-(IV) in one call.  scores_out (optional, [batch][n_kv_heads][N] fp32)
+ * receives the final scores s^(T). */
+graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, const void *K,
+                                const void *V, void *K_out, void *V_out, int32_t *idx_out,
+                                float *scores_out, void *workspace, size_t workspace_bytes,
+                                void *stream);
+
+/* Synchronises `stream` and returns the status word kernels keep at the head of the workspace
+ * (GRAPHKV_OK unless a bounded device-side wait ran out or a CUDA error surfaced).  The only
+ * call that blocks the host. */
+graphkv_status graphkv_read_status(const void *workspace, void *stream);
+
+const char *graphkv_status_string(graphkv_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRAPHKV_H_ */

@@ -1,0 +1,186 @@
+"""ctypes binding of libgraphkv.so: argument marshalling only.
+
+Every function takes CUDA torch tensors, fills a `graphkv_params` struct from their shapes and
+strides, and passes raw device pointers plus the current CUDA stream to the C entry point of
+the same name (declared in include/graphkv.h).  No step of the path runs here, and there is no
+CPU route: loading fails loudly if the CUDA library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libgraphkv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+BF16, F32 = 0, 1
+
+EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_score",
+           "graphkv_propagate", "graphkv_select_gather", "graphkv_compress",
+           "graphkv_read_status", "graphkv_status_string")
+
+
+class GraphKVError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class Params(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("seq_len", C.c_int32), ("window", C.c_int32),
+                ("budget", C.c_int32), ("pool_kernel", C.c_int32), ("pool_mode", C.c_int32),
+                ("topk_nodes", C.c_int32), ("neighbors", C.c_int32), ("rounds", C.c_int32),
+                ("decay", C.c_float), ("dtype", C.c_int32),
+                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
+                ("v_stride", C.c_int64 * 3)]
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """The loaded CUDA library.  Raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2509_00388_b200.build` "
+                "(nvcc, sm_100a).  This library has no CPU or PyTorch fallback.")
+        L = C.CDLL(LIB_PATH)
+        P = C.POINTER(Params)
+        vp, sz = C.c_void_p, C.c_size_t
+        L.graphkv_workspace_bytes.restype = sz
+        L.graphkv_workspace_bytes.argtypes = [P]
+        L.graphkv_resolve_neighbors.restype = C.c_int32
+        L.graphkv_resolve_neighbors.argtypes = [C.c_int32, C.c_int32]
+        L.graphkv_score.restype = C.c_int
+        L.graphkv_score.argtypes = [P, vp, vp, vp, vp, sz, vp]
+        L.graphkv_propagate.restype = C.c_int
+        L.graphkv_propagate.argtypes = [P, vp, vp, vp, vp, sz, vp]
+        L.graphkv_select_gather.restype = C.c_int
+        L.graphkv_select_gather.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.graphkv_compress.restype = C.c_int
+        L.graphkv_compress.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.graphkv_read_status.restype = C.c_int
+        L.graphkv_read_status.argtypes = [vp, vp]
+        L.graphkv_status_string.restype = C.c_char_p
+        L.graphkv_status_string.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().graphkv_status_string(int(code)).decode()
+
+
+def resolve_neighbors(n_prefix: int, neighbors: int) -> int:
+    return int(lib().graphkv_resolve_neighbors(n_prefix, neighbors))
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _strides3(t: Optional[torch.Tensor]):
+    if t is None:
+        return (C.c_int64 * 3)(0, 0, 128)
+    assert t.dim() == 4 and t.stride(3) == 1, "expected [batch, heads, rows, D] with D contiguous"
+    return (C.c_int64 * 3)(t.stride(0), t.stride(1), t.stride(2))
+
+
+def make_params(K: torch.Tensor, *, window: int, n_q_heads: Optional[int] = None,
+                Qw: Optional[torch.Tensor] = None, V: Optional[torch.Tensor] = None,
+                budget: int = 1, pool_kernel: int = 1, topk_nodes: int = 0, neighbors: int = 0,
+                rounds: int = 0, decay: float = 1.0) -> Params:
+    b, hkv, ell, d = K.shape
+    hq = Qw.shape[1] if Qw is not None else (n_q_heads or hkv)
+    p = Params()
+    p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = b, hq, hkv, d
+    p.seq_len, p.window, p.budget = ell, window, budget
+    p.pool_kernel, p.pool_mode = pool_kernel, 0
+    p.topk_nodes, p.neighbors, p.rounds, p.decay = topk_nodes, neighbors, rounds, decay
+    p.dtype = _dtype_code(K)
+    p.q_stride = _strides3(Qw)
+    p.k_stride = _strides3(K)
+    p.v_stride = _strides3(V if V is not None else K)
+    return p
+
+
+def workspace_bytes(p: Params) -> int:
+    return int(lib().graphkv_workspace_bytes(C.byref(p)))
+
+
+def alloc_workspace(p: Params, device) -> torch.Tensor:
+    n = workspace_bytes(p)
+    if n == 0:
+        raise GraphKVError(ERR_INVALID_ARG, "graphkv_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise GraphKVError(code, where)
+
+
+def graphkv_score(p: Params, Qw: torch.Tensor, K: torch.Tensor, scores: torch.Tensor,
+                  ws: torch.Tensor) -> None:
+    _check(lib().graphkv_score(C.byref(p), _ptr(Qw), _ptr(K), _ptr(scores), _ptr(ws),
+                               ws.numel(), _stream(K.device)), "graphkv_score")
+
+
+def graphkv_propagate(p: Params, K: torch.Tensor, scores: torch.Tensor,
+                      src_idx_out: Optional[torch.Tensor], ws: torch.Tensor) -> None:
+    _check(lib().graphkv_propagate(C.byref(p), _ptr(K), _ptr(scores), _ptr(src_idx_out),
+                                   _ptr(ws), ws.numel(), _stream(K.device)),
+           "graphkv_propagate")
+
+
+def graphkv_select_gather(p: Params, scores: torch.Tensor, K: Optional[torch.Tensor],
+                          V: Optional[torch.Tensor], K_out: Optional[torch.Tensor],
+                          V_out: Optional[torch.Tensor], idx_out: torch.Tensor,
+                          ws: torch.Tensor) -> None:
+    _check(lib().graphkv_select_gather(C.byref(p), _ptr(scores), _ptr(K), _ptr(V), _ptr(K_out),
+                                       _ptr(V_out), _ptr(idx_out), _ptr(ws), ws.numel(),
+                                       _stream(scores.device)), "graphkv_select_gather")
+
+
+def graphkv_compress(p: Params, Qw: torch.Tensor, K: torch.Tensor, V: torch.Tensor,
+                     K_out: torch.Tensor, V_out: torch.Tensor, idx_out: torch.Tensor,
+                     scores_out: Optional[torch.Tensor], ws: torch.Tensor) -> None:
+    _check(lib().graphkv_compress(C.byref(p), _ptr(Qw), _ptr(K), _ptr(V), _ptr(K_out),
+                                  _ptr(V_out), _ptr(idx_out), _ptr(scores_out), _ptr(ws),
+                                  ws.numel(), _stream(K.device)), "graphkv_compress")
+
+
+def graphkv_read_status(ws: torch.Tensor) -> int:
+    return int(lib().graphkv_read_status(_ptr(ws), _stream(ws.device)))
+
+
+def alloc_outputs(p: Params, like: torch.Tensor, want_scores: bool = True
+                  ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor, Optional[torch.Tensor]]:
+    """Dense output tensors of the shapes the C ABI writes."""
+    n = p.seq_len - p.window
+    shape = (p.batch, p.n_kv_heads, p.budget + p.window, p.head_dim)
+    K_out = torch.empty(shape, dtype=like.dtype, device=like.device)
+    V_out = torch.empty(shape, dtype=like.dtype, device=like.device)
+    idx = torch.empty((p.batch, p.n_kv_heads, p.budget), dtype=torch.int32, device=like.device)
+    s = (torch.empty((p.batch, p.n_kv_heads, n), dtype=torch.float32, device=like.device)
+         if want_scores else None)
+    return K_out, V_out, idx, s

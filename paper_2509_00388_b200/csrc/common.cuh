@@ -1,0 +1,64 @@
+// Shared device/host helpers of the GraphKV CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "graphkv.h"
+
+namespace graphkv {
+
+constexpr int kHeadDim = 128;          // D, fixed by the library
+constexpr int kMaxRows = 256;          // G*W limit (one TMEM accumulator tile of query rows)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegBig = -1.0e30f;    // finite stand-in for -inf in running maxima
+constexpr float kNormEps = 1e-12f;     // floor of a key norm in Eq. 1
+
+// Shape of one call, resolved once on the host and passed by value to kernels.
+struct Dims {
+    int batch, hq, hkv, G, W, N, L, GW;
+    int B, kp, K_src, m, T;
+    float lambda;
+    int units;                 // batch * hkv independent (sequence, KV head) problems
+    long long qs[3], ks[3], vs[3];
+};
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// ---- element access: 8 consecutive elements of a row as fp32 --------------------------------
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8])
+{
+    const uint4 raw = *reinterpret_cast<const uint4 *>(p);
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+__device__ __forceinline__ void load8(const float *p, float (&v)[8])
+{
+    const float4 a = *reinterpret_cast<const float4 *>(p);
+    const float4 b = *reinterpret_cast<const float4 *>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+// Order-preserving map fp32 -> uint32 (larger float <=> larger key); -0 and +0 map to one key.
+__device__ __forceinline__ uint32_t float_to_key(float x)
+{
+    uint32_t u = __float_as_uint(x);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+}  // namespace graphkv

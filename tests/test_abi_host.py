@@ -1,0 +1,106 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2509_00388_b200 import binding as gk
+from paper_2509_00388_b200 import build as gk_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    gk_build.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "graphkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(graphkv_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert set(names) >= {"graphkv_score", "graphkv_propagate", "graphkv_select_gather",
+                          "graphkv_compress", "graphkv_workspace_bytes"}
+    lib = C.CDLL(gk.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in graphkv.h but not exported"
+    assert set(gk.EXPORTS) == set(names)
+
+
+def test_params_struct_matches_header_size():
+    # 14 four-byte fields + 9 int64 strides
+    assert C.sizeof(gk.Params) == 14 * 4 + 9 * 8
+
+
+def _params(**kw):
+    K = torch.empty(1, 2, 104, 128, dtype=torch.bfloat16)
+    Q = torch.empty(1, 4, 4, 128, dtype=torch.bfloat16)
+    base = dict(window=4, budget=10, pool_kernel=7, topk_nodes=3, neighbors=2, rounds=1, decay=1.0)
+    base.update(kw)
+    return gk.make_params(K, Qw=Q, V=K, **base)
+
+
+def test_workspace_bytes_positive_and_monotone():
+    a = gk.workspace_bytes(_params())
+    b = gk.workspace_bytes(_params(topk_nodes=30))
+    assert a > 0 and b > a and a % 256 == 0
+
+
+@pytest.mark.parametrize("bad", [
+    dict(budget=0), dict(budget=101), dict(pool_kernel=4), dict(pool_kernel=0),
+    dict(topk_nodes=-1), dict(topk_nodes=101), dict(neighbors=100), dict(rounds=-1),
+    dict(decay=1.5), dict(decay=-0.1), dict(decay=float("nan")),
+])
+def test_invalid_params_are_rejected_on_the_host(bad):
+    p = _params(**bad)
+    assert gk.workspace_bytes(p) == 0
+    rc = gk.lib().graphkv_compress(C.byref(p), 16, 16, 16, 16, 16, 16, None, 256, 1 << 30, None)
+    assert rc == gk.ERR_INVALID_ARG
+
+
+def test_unsupported_shapes():
+    p = _params()
+    p.head_dim = 64
+    assert gk.lib().graphkv_score(C.byref(p), 16, 16, 16, 256, 1 << 30, None) == gk.ERR_UNSUPPORTED
+    p = _params()
+    p.n_q_heads, p.window, p.seq_len = 64, 64, 164      # G*W = 2048 rows
+    assert gk.lib().graphkv_score(C.byref(p), 16, 16, 16, 256, 1 << 30, None) == gk.ERR_UNSUPPORTED
+    p = _params()
+    p.n_q_heads = 5                                       # not a multiple of the KV heads
+    assert gk.lib().graphkv_score(C.byref(p), 16, 16, 16, 256, 1 << 30, None) == gk.ERR_INVALID_ARG
+
+
+def test_null_pointers_misalignment_and_workspace():
+    p = _params()
+    need = gk.workspace_bytes(p)
+    L = gk.lib()
+    assert L.graphkv_score(C.byref(p), None, 16, 16, 256, need, None) == gk.ERR_INVALID_ARG
+    assert L.graphkv_score(C.byref(p), 16, 24, 16, 256, need, None) == gk.ERR_INVALID_ARG
+    assert L.graphkv_score(C.byref(p), 16, 16, 16, None, need, None) == gk.ERR_WORKSPACE
+    assert L.graphkv_score(C.byref(p), 16, 16, 16, 256, need - 1, None) == gk.ERR_WORKSPACE
+    assert L.graphkv_score(C.byref(p), 16, 16, 16, 128, need, None) == gk.ERR_WORKSPACE
+    assert L.graphkv_select_gather(C.byref(p), 16, 16, None, None, None, 16, 256, need,
+                                   None) == gk.ERR_INVALID_ARG       # K without K_out
+    p.k_stride[2] = 100                                                 # rows would overlap
+    assert L.graphkv_score(C.byref(p), 16, 16, 16, 256, need, None) == gk.ERR_INVALID_ARG
+
+
+def test_status_strings_and_neighbour_rule():
+    assert gk.status_string(gk.OK) == "ok"
+    assert "workspace" in gk.status_string(gk.ERR_WORKSPACE)
+    assert [gk.resolve_neighbors(n, 0) for n in (512, 16384, 32768, 131072)] == [1, 16, 32, 32]
+    assert gk.resolve_neighbors(5, 0) == 1 and gk.resolve_neighbors(1, 0) == 0
+    assert gk.resolve_neighbors(32768, 7) == 7
+
+
+def test_binding_has_no_cpu_route():
+    import inspect
+    src = inspect.getsource(gk)
+    assert "oracle" not in src

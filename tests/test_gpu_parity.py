@@ -1,0 +1,233 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs, stage by stage and end to end."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import graphkv_oracle as okv
+from paper_2509_00388_b200 import workloads as wl
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gk():
+    from paper_2509_00388_b200 import binding
+    binding.lib()
+    return binding
+
+
+def run_staged(gk, Qw, K, V, **kw):
+    """score -> propagate -> select_gather on cuda:0; returns CPU copies of every stage."""
+    dev = torch.device("cuda:0")
+    Qd, Kd, Vd = Qw.to(dev), K.to(dev), V.to(dev)
+    p = gk.make_params(Kd, Qw=Qd, V=Vd, **kw)
+    ws = gk.alloc_workspace(p, dev)
+    K_out, V_out, idx, s = gk.alloc_outputs(p, Kd)
+    gk.graphkv_score(p, Qd, Kd, s, ws)
+    out = {"scores0": s.cpu()}
+    src = None
+    if kw.get("topk_nodes", 0) > 0:
+        src = torch.empty((p.batch, p.n_kv_heads, p.topk_nodes), dtype=torch.int32, device=dev)
+    gk.graphkv_propagate(p, Kd, s, src, ws)
+    if src is not None:
+        out["src"] = src.cpu()
+    out["scores"] = s.cpu()
+    gk.graphkv_select_gather(p, s, Kd, Vd, K_out, V_out, idx, ws)
+    assert gk.graphkv_read_status(ws) == gk.OK
+    out.update(idx=idx.cpu(), K_out=K_out.cpu(), V_out=V_out.cpu())
+    return out
+
+
+def run_fused(gk, Qw, K, V, **kw):
+    dev = torch.device("cuda:0")
+    Qd, Kd, Vd = Qw.to(dev), K.to(dev), V.to(dev)
+    p = gk.make_params(Kd, Qw=Qd, V=Vd, **kw)
+    ws = gk.alloc_workspace(p, dev)
+    K_out, V_out, idx, s = gk.alloc_outputs(p, Kd)
+    gk.graphkv_compress(p, Qd, Kd, Vd, K_out, V_out, idx, s, ws)
+    assert gk.graphkv_read_status(ws) == gk.OK
+    return {"idx": idx.cpu(), "K_out": K_out.cpu(), "V_out": V_out.cpu(), "scores": s.cpu()}
+
+
+def cfg_kwargs(cfg, layer=0):
+    return dict(window=cfg.window, budget=cfg.layer_budget(layer), pool_kernel=cfg.pool_kernel,
+                topk_nodes=cfg.topk_nodes, neighbors=cfg.neighbors, rounds=cfg.rounds,
+                decay=cfg.decay)
+
+
+def check(gk, cfg, layer=0, sequences=None, strict_overlap=True, **override):
+    inp = wl.make_inputs(cfg, layer=layer, sequences=sequences)
+    kw = cfg_kwargs(cfg, layer)
+    kw.update(override)
+    staged = run_staged(gk, inp["Qw"], inp["K"], inp["V"], **kw)
+    fused = run_fused(gk, inp["Qw"], inp["K"], inp["V"], **kw)
+    for name in ("idx", "K_out", "V_out", "scores"):
+        assert torch.equal(staged[name].view(torch.uint8), fused[name].view(torch.uint8)), \
+            f"fused compress differs from the staged calls in {name}"
+    rep = pu.check_compress(staged, inp["Qw"], inp["K"], inp["V"], strict_overlap=strict_overlap,
+                            **kw)
+    print(json.dumps({"config": cfg.name, "layer": layer, **rep.as_dict()}))
+    return rep
+
+
+# ---- config 1: the tiny fp32 single head, with the neighbour sweep ------------------------------
+@pytest.mark.parametrize("m", [0, 1, 4, 16])
+@pytest.mark.parametrize("lam", [1.0, 0.5, 0.25])
+def test_tiny_fp32_config(gk, m, lam):
+    check(gk, wl.TINY, neighbors=m, decay=lam)
+
+
+# ---- reduced copies of the large configs: several tiles and a ragged tail ----------------------
+SMALL = [
+    dict(n_prefix=5000, budget=300, n_q_heads=8, n_kv_heads=2, neighbors=8),
+    dict(n_prefix=4097, budget=64, n_q_heads=4, n_kv_heads=4, window=32, topk_nodes=5),
+    dict(n_prefix=3000, budget=500, n_q_heads=8, n_kv_heads=2, window=64, topk_nodes=32, rounds=4),
+    dict(n_prefix=2049, budget=100, n_q_heads=4, n_kv_heads=1, window=17, batch=3, neighbors=3),
+    dict(n_prefix=1024, budget=1024, n_q_heads=2, n_kv_heads=2, window=8),
+]
+
+
+@pytest.mark.parametrize("i", range(len(SMALL)))
+def test_reduced_bf16_configs(gk, i):
+    cfg = wl.scaled(wl.LLAMA_32K, n_clusters=32, **SMALL[i])
+    check(gk, cfg, strict_overlap=False)
+
+
+def test_reduced_fp32_multihead(gk):
+    cfg = wl.scaled(wl.LLAMA_32K, dtype="f32", n_prefix=2500, budget=200, n_q_heads=8,
+                    n_kv_heads=2, n_clusters=32, neighbors=6)
+    check(gk, cfg, strict_overlap=False)
+
+
+# ---- degenerate and edge cases ----------------------------------------------------------------
+@pytest.mark.parametrize("case", [
+    dict(n_prefix=40, budget=7, topk_nodes=3, neighbors=2),            # N below every tile size
+    dict(n_prefix=1, budget=1, topk_nodes=1, neighbors=0),             # single node, m = 0
+    dict(n_prefix=2, budget=1, topk_nodes=2, neighbors=1),
+    dict(n_prefix=333, budget=333, topk_nodes=4, neighbors=5),         # keep everything
+    dict(n_prefix=333, budget=1, topk_nodes=333, neighbors=1),         # every node a source
+    dict(n_prefix=600, budget=50, topk_nodes=0, neighbors=0),          # no sources
+    dict(n_prefix=600, budget=50, topk_nodes=4, neighbors=0, rounds=0),  # T = 0: base method
+    dict(n_prefix=600, budget=50, topk_nodes=4, neighbors=7, pool_kernel=1),
+    dict(n_prefix=600, budget=50, topk_nodes=2, neighbors=599),        # m = N - 1
+    dict(n_prefix=600, budget=50, topk_nodes=4, neighbors=7, decay=0.0),
+    dict(n_prefix=700, budget=50, topk_nodes=4, neighbors=7, pool_kernel=31),
+])
+def test_edge_cases(gk, case):
+    cfg = wl.scaled(wl.LLAMA_32K, n_q_heads=4, n_kv_heads=2, n_clusters=8, **case)
+    check(gk, cfg, strict_overlap=False)
+
+
+def test_zero_queries_give_constant_scores_and_lowest_indices(gk):
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=3000, budget=77, n_q_heads=4, n_kv_heads=2, rounds=0)
+    inp = wl.make_inputs(cfg)
+    Qw = torch.zeros_like(inp["Qw"])
+    out = run_fused(gk, Qw, inp["K"], inp["V"], **cfg_kwargs(cfg))
+    expect = cfg.group * sum(1.0 / (cfg.n_prefix + r + 1) for r in range(cfg.window))
+    assert pu.score_rel_err(out["scores"], torch.full_like(out["scores"], expect)) < 1e-5
+    assert torch.equal(out["idx"], torch.arange(77, dtype=torch.int32).expand(1, 2, 77))
+
+
+def test_exact_duplicate_keys_tie_break_like_the_oracle(gk):
+    # bit-identical keys give bit-identical cosines: the lower index must win on both sides
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=2000, budget=100, n_q_heads=4, n_kv_heads=1,
+                    n_clusters=8, dup_sigma=0.0, dup_frac=0.5, neighbors=16)
+    check(gk, cfg, strict_overlap=False)
+
+
+def test_strided_inputs(gk):
+    # K and V as views of a [batch, L, heads, D] buffer (token-major, the layout of a fused
+    # QKV projection): strides are not those of a dense [b, h, L, D] tensor
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=1500, budget=100, n_q_heads=8, n_kv_heads=2,
+                    n_clusters=16, batch=2)
+    inp = wl.make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    kw = cfg_kwargs(cfg)
+    dense = run_fused(gk, inp["Qw"], inp["K"], inp["V"], **kw)
+    Kt = inp["K"].to(dev).permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    Vt = inp["V"].to(dev).permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    Qd = inp["Qw"].to(dev)
+    assert not Kt.is_contiguous()
+    p = gk.make_params(Kt, Qw=Qd, V=Vt, **kw)
+    ws = gk.alloc_workspace(p, dev)
+    K_out, V_out, idx, s = gk.alloc_outputs(p, Kt)
+    gk.graphkv_compress(p, Qd, Kt, Vt, K_out, V_out, idx, s, ws)
+    assert torch.equal(idx.cpu(), dense["idx"])
+    assert torch.equal(K_out.cpu().view(torch.int16), dense["K_out"].view(torch.int16))
+    assert torch.equal(V_out.cpu().view(torch.int16), dense["V_out"].view(torch.int16))
+    assert torch.equal(s.cpu(), dense["scores"])
+
+
+def test_runs_are_bitwise_repeatable(gk):
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=6000, budget=256, n_q_heads=8, n_kv_heads=2)
+    inp = wl.make_inputs(cfg)
+    a = run_fused(gk, inp["Qw"], inp["K"], inp["V"], **cfg_kwargs(cfg))
+    b = run_fused(gk, inp["Qw"], inp["K"], inp["V"], **cfg_kwargs(cfg))
+    for name in a:
+        assert torch.equal(a[name].view(torch.uint8), b[name].view(torch.uint8))
+
+
+def test_select_gather_alone_is_bit_exact_with_planted_ties(gk):
+    dev = torch.device("cuda:0")
+    for n, B, seed in [(5000, 300, 0), (131072, 4096, 1), (33, 33, 2), (1025, 1, 3)]:
+        s = wl.make_scores(3, n, seed, tie_frac=0.3).reshape(1, 3, n)
+        cfg = wl.scaled(wl.LLAMA_32K, n_prefix=n, budget=B, n_q_heads=3, n_kv_heads=3, window=4)
+        inp = wl.make_inputs(cfg)
+        Kd, Vd = inp["K"].to(dev), inp["V"].to(dev)
+        p = gk.make_params(Kd, V=Vd, window=4, budget=B)
+        ws = gk.alloc_workspace(p, dev)
+        K_out, V_out, idx, _ = gk.alloc_outputs(p, Kd, want_scores=False)
+        gk.graphkv_select_gather(p, s.to(dev), Kd, Vd, K_out, V_out, idx, ws)
+        oK, oV, oidx = okv.select_gather(s, inp["K"], inp["V"], 4, B)
+        assert torch.equal(idx.cpu(), oidx)
+        assert torch.equal(K_out.cpu().view(torch.int16), oK.view(torch.int16))
+        assert torch.equal(V_out.cpu().view(torch.int16), oV.view(torch.int16))
+
+
+def test_propagate_alone_from_oracle_scores(gk):
+    # teacher forcing the other way: the GPU stage starts from the oracle's fp32 scores
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=7000, budget=256, n_q_heads=8, n_kv_heads=2,
+                    n_clusters=64)
+    inp = wl.make_inputs(cfg)
+    s0 = okv.score(inp["Qw"], inp["K"], cfg.window, cfg.pool_kernel)
+    o_s, o_src = okv.propagate(inp["K"], s0, cfg.window, cfg.topk_nodes, cfg.neighbors,
+                               cfg.rounds, cfg.decay)
+    dev = torch.device("cuda:0")
+    Kd = inp["K"].to(dev)
+    p = gk.make_params(Kd, n_q_heads=cfg.n_q_heads, **cfg_kwargs(cfg))
+    ws = gk.alloc_workspace(p, dev)
+    s = s0.to(dev)
+    src = torch.empty((1, 2, cfg.topk_nodes), dtype=torch.int32, device=dev)
+    gk.graphkv_propagate(p, Kd, s, src, ws)
+    assert torch.equal(torch.sort(src.cpu(), dim=-1).values.int(),
+                       torch.sort(o_src, dim=-1).values.int())
+    assert pu.score_rel_err(s.cpu(), o_s) <= pu.SCORE_RTOL
+
+
+# ---- the benchmark configurations at full size -------------------------------------------------
+def test_full_llama_32k(gk):
+    rep = check(gk, wl.LLAMA_32K)
+    assert rep.overlap >= pu.MIN_OVERLAP
+
+
+@pytest.mark.parametrize("layer", [0, 13, 31])
+def test_full_mistral_16k_layers(gk, layer):
+    check(gk, wl.MISTRAL_16K, layer=layer)
+
+
+@pytest.mark.parametrize("layer", [0, 16, 31])
+def test_full_pyramid_budgets(gk, layer):
+    cfg = wl.PYRAMID_32K
+    assert cfg.layer_budget(0) == 2048 and cfg.layer_budget(31) == 128
+    check(gk, cfg, layer=layer)
+
+
+def test_full_long_context_128k(gk):
+    # all four sequences of the batch, two at a time to bound host memory
+    for seqs in ([0, 1], [2, 3]):
+        check(gk, wl.LONG_128K, sequences=seqs)
