@@ -123,6 +123,21 @@ graphkv_status graphkv_read_status(const void *workspace, void *stream);
 
 const char *graphkv_status_string(graphkv_status status);
 
+/* ---- tracing (the paper has no counterpart: measurement support of this library) -------------
+ * graphkv_launch_count: kernels this process has launched through the library so far.
+ * graphkv_trace_enable(1): from now on every kernel launch is bracketed by a pair of CUDA events
+ * recorded on the launch's stream (host-side objects; no device memory).  Off by default.
+ * graphkv_trace_read: waits for the recorded events, writes up to `capacity` records (kernel
+ * name, device milliseconds) in launch order, forgets all records and returns how many were
+ * written.  Not to be called while a traced stream is being captured into a CUDA graph. */
+typedef struct {
+    char name[40];
+    float ms;
+} graphkv_trace_record;
+int64_t graphkv_launch_count(void);
+void graphkv_trace_enable(int32_t enable);
+int32_t graphkv_trace_read(graphkv_trace_record *out, int32_t capacity);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,8 @@ BF16, F32 = 0, 1
 
 EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_score",
            "graphkv_propagate", "graphkv_select_gather", "graphkv_compress",
-           "graphkv_read_status", "graphkv_status_string")
+           "graphkv_read_status", "graphkv_status_string", "graphkv_launch_count",
+           "graphkv_trace_enable", "graphkv_trace_read")
 
 
 class GraphKVError(RuntimeError):
@@ -38,6 +39,10 @@ class Params(C.Structure):
                 ("decay", C.c_float), ("dtype", C.c_int32),
                 ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
                 ("v_stride", C.c_int64 * 3)]
+
+
+class TraceRecord(C.Structure):
+    _fields_ = [("name", C.c_char * 40), ("ms", C.c_float)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -70,6 +75,12 @@ def lib() -> C.CDLL:
         L.graphkv_read_status.argtypes = [vp, vp]
         L.graphkv_status_string.restype = C.c_char_p
         L.graphkv_status_string.argtypes = [C.c_int]
+        L.graphkv_launch_count.restype = C.c_int64
+        L.graphkv_launch_count.argtypes = []
+        L.graphkv_trace_enable.restype = None
+        L.graphkv_trace_enable.argtypes = [C.c_int32]
+        L.graphkv_trace_read.restype = C.c_int32
+        L.graphkv_trace_read.argtypes = [C.POINTER(TraceRecord), C.c_int32]
         _lib = L
     return _lib
 
@@ -171,6 +182,21 @@ def graphkv_compress(p: Params, Qw: torch.Tensor, K: torch.Tensor, V: torch.Tens
 
 def graphkv_read_status(ws: torch.Tensor) -> int:
     return int(lib().graphkv_read_status(_ptr(ws), _stream(ws.device)))
+
+
+def graphkv_launch_count() -> int:
+    return int(lib().graphkv_launch_count())
+
+
+def graphkv_trace_enable(enable: bool) -> None:
+    lib().graphkv_trace_enable(1 if enable else 0)
+
+
+def graphkv_trace_read(capacity: int = 1 << 16):
+    """[(kernel name, device ms), ...] of the launches traced since the last read."""
+    buf = (TraceRecord * capacity)()
+    n = lib().graphkv_trace_read(buf, capacity)
+    return [(buf[i].name.decode(), float(buf[i].ms)) for i in range(n)]
 
 
 def alloc_outputs(p: Params, like: torch.Tensor, want_scores: bool = True

@@ -1,6 +1,10 @@
 // C ABI of the GraphKV library: argument validation, workspace layout and kernel launches.
+#include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "common.cuh"
 #include "gather.cuh"
@@ -106,6 +110,42 @@ inline graphkv_status launch_status()
     return GRAPHKV_OK;
 }
 
+// ---- launch accounting and optional per-kernel timing -----------------------------------------
+std::atomic<long long> g_launches{0};
+std::atomic<int> g_trace_on{0};
+std::mutex g_trace_mu;
+struct TraceEntry { const char *name; cudaEvent_t start, stop; };
+std::vector<TraceEntry> g_trace;
+
+// Counts one kernel launch; with tracing on, brackets it with CUDA events on its stream.
+struct LaunchScope {
+    cudaStream_t st;
+    bool traced;
+    TraceEntry e;
+    LaunchScope(const char *name, cudaStream_t s) : st(s), traced(false)
+    {
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (!g_trace_on.load(std::memory_order_relaxed)) return;
+        e.name = name;
+        if (cudaEventCreate(&e.start) != cudaSuccess) return;
+        if (cudaEventCreate(&e.stop) != cudaSuccess) { cudaEventDestroy(e.start); return; }
+        cudaEventRecord(e.start, st);
+        traced = true;
+    }
+    ~LaunchScope()
+    {
+        if (!traced) return;
+        cudaEventRecord(e.stop, st);
+        std::lock_guard<std::mutex> lk(g_trace_mu);
+        g_trace.push_back(e);
+    }
+};
+#define GKV_LAUNCH(name, st, ...)        \
+    do {                                 \
+        LaunchScope _scope(name, st);    \
+        __VA_ARGS__;                     \
+    } while (0)
+
 template <typename T> inline T *at(void *ws, size_t off)
 {
     return reinterpret_cast<T *>(static_cast<unsigned char *>(ws) + off);
@@ -119,8 +159,9 @@ graphkv_status run_score(const Dims &d, const Layout &l, const T *Q, const T *K,
     float *part = at<float>(ws, l.part);
     float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
     const int threads = ceil_div(d.GW, 32) * 32;
-    score_stats_simt<T><<<dim3(l.n_stat_chunks, d.units), threads, 0, st>>>(
-        d, Q, K, part, l.n_stat_chunks, at<int>(ws, l.status));
+    GKV_LAUNCH("score_stats_simt", st,
+               (score_stats_simt<T><<<dim3(l.n_stat_chunks, d.units), threads, 0, st>>>(
+                   d, Q, K, part, l.n_stat_chunks, at<int>(ws, l.status))));
     const size_t smem = ((size_t)d.GW * kHeadDim + 2 * d.GW) * sizeof(float);
     static bool attr_set[2] = {false, false};
     if (!attr_set[sizeof(T) == 2]) {
@@ -130,10 +171,13 @@ graphkv_status run_score(const Dims &d, const Layout &l, const T *Q, const T *K,
             return GRAPHKV_ERR_CUDA;
         attr_set[sizeof(T) == 2] = true;
     }
-    score_emit_simt<T><<<dim3(ceil_div(d.N, kEmitChunk), d.units), kEmitThreads, smem, st>>>(
-        d, Q, K, part, l.n_stat_chunks, a);
+    GKV_LAUNCH("score_emit_simt", st,
+               (score_emit_simt<T><<<dim3(ceil_div(d.N, kEmitChunk), d.units), kEmitThreads, smem,
+                                     st>>>(d, Q, K, part, l.n_stat_chunks, a)));
     if (d.kp > 1)
-        pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a, scores);
+        GKV_LAUNCH("pool_max", st,
+                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a,
+                                                                                      scores)));
     return launch_status();
 }
 
@@ -145,15 +189,18 @@ graphkv_status run_propagate(const Dims &d, const Layout &l, const T *K, float *
     if (d.K_src == 0) return GRAPHKV_OK;
     int *src = src_out ? src_out : at<int>(ws, l.src);
     SelectArgs sa{scores, d.N, d.N, d.K_src, nullptr, src, nullptr};
-    topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa);
+    GKV_LAUNCH("select_sources", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
     if (d.T == 0 || d.m == 0) return launch_status();
     float *sims = at<float>(ws, l.sims);
-    similarity_simt<T><<<dim3(ceil_div(d.N, kSimChunk), d.units), kSimThreads, 0, st>>>(d, K, src,
-                                                                                      sims);
+    GKV_LAUNCH("similarity_simt", st,
+               (similarity_simt<T><<<dim3(ceil_div(d.N, kSimChunk), d.units), kSimThreads, 0, st>>>(
+                   d, K, src, sims)));
     SelectArgs na{sims, d.N, d.N, d.m, src, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e)};
-    topk_select_kernel<<<d.units * d.K_src, kSelectThreads, 0, st>>>(na);
-    decay_rounds_kernel<<<d.units, 256, 0, st>>>(d, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e),
-                                                scores);
+    GKV_LAUNCH("select_neighbors", st,
+               (topk_select_kernel<<<d.units * d.K_src, kSelectThreads, 0, st>>>(na)));
+    GKV_LAUNCH("decay_rounds", st,
+               (decay_rounds_kernel<<<d.units, 256, 0, st>>>(d, at<int>(ws, l.nbr_idx),
+                                                             at<float>(ws, l.nbr_e), scores)));
     return launch_status();
 }
 
@@ -163,15 +210,16 @@ graphkv_status run_select_gather(const Dims &d, int elem_bytes, const float *sco
                                  cudaStream_t st)
 {
     SelectArgs sa{scores, d.N, d.N, d.B, nullptr, idx_out, nullptr};
-    topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa);
+    GKV_LAUNCH("select_budget", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
     if (K || V) {
         const long long total = (long long)d.units * (d.B + d.W) * (kHeadDim * elem_bytes / 16);
         const int blocks = (int)std::min<long long>((total + kGatherThreads - 1) / kGatherThreads,
                                                     148LL * 16);
-        gather_rows_kernel<<<blocks, kGatherThreads, 0, st>>>(
-            d, elem_bytes, static_cast<const unsigned char *>(K),
-            static_cast<const unsigned char *>(V), idx_out, static_cast<unsigned char *>(K_out),
-            static_cast<unsigned char *>(V_out));
+        GKV_LAUNCH("gather_rows", st,
+                   (gather_rows_kernel<<<blocks, kGatherThreads, 0, st>>>(
+                       d, elem_bytes, static_cast<const unsigned char *>(K),
+                       static_cast<const unsigned char *>(V), idx_out,
+                       static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out))));
     }
     return launch_status();
 }
@@ -291,6 +339,33 @@ graphkv_status graphkv_read_status(const void *workspace, void *stream)
     if (cudaStreamSynchronize(st) != cudaSuccess) return GRAPHKV_ERR_CUDA;
     if (word < 0 || word > GRAPHKV_ERR_TIMEOUT) return GRAPHKV_ERR_CUDA;
     return static_cast<graphkv_status>(word);
+}
+
+int64_t graphkv_launch_count(void) { return g_launches.load(); }
+
+void graphkv_trace_enable(int32_t enable)
+{
+    g_trace_on.store(enable ? 1 : 0);
+}
+
+int32_t graphkv_trace_read(graphkv_trace_record *out, int32_t capacity)
+{
+    std::lock_guard<std::mutex> lk(g_trace_mu);
+    int32_t n = 0;
+    for (const TraceEntry &e : g_trace) {
+        float ms = -1.f;
+        if (cudaEventSynchronize(e.stop) == cudaSuccess) cudaEventElapsedTime(&ms, e.start, e.stop);
+        if (out && n < capacity) {
+            strncpy(out[n].name, e.name, sizeof(out[n].name) - 1);
+            out[n].name[sizeof(out[n].name) - 1] = 0;
+            out[n].ms = ms;
+            ++n;
+        }
+        cudaEventDestroy(e.start);
+        cudaEventDestroy(e.stop);
+    }
+    g_trace.clear();
+    return n;
 }
 
 const char *graphkv_status_string(graphkv_status status)
