@@ -1,4 +1,5 @@
 // C ABI of the GraphKV library: argument validation, workspace layout and kernel launches.
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
@@ -10,6 +11,7 @@
 #include "gather.cuh"
 #include "propagate_simt.cuh"
 #include "score_simt.cuh"
+#include "score_tc.cuh"
 #include "select.cuh"
 
 using namespace graphkv;
@@ -30,7 +32,8 @@ struct Layout {
     size_t nbr_idx;     // neighbourhoods [units][K_src][m]
     size_t nbr_e;
     size_t total;
-    int n_stat_chunks;
+    int n_stat_chunks;  // key chunks of the SIMT statistics sweep
+    int max_parts;      // partial statistics per row the region can hold
 };
 
 graphkv_status resolve(const graphkv_params *p, Dims *d)
@@ -78,8 +81,9 @@ Layout layout_of(const Dims &d)
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     l.n_stat_chunks = ceil_div(d.L, kStatsChunk);
+    l.max_parts = l.n_stat_chunks > 2 * 148 ? l.n_stat_chunks : 2 * 148;
     l.status = take(kAlign);
-    l.part = take((size_t)d.units * l.n_stat_chunks * d.GW * 2 * sizeof(float));
+    l.part = take((size_t)d.units * l.max_parts * d.GW * 2 * sizeof(float));
     l.a = take((size_t)d.units * d.N * sizeof(float));
     l.s = take((size_t)d.units * d.N * sizeof(float));
     l.src = take((size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * sizeof(int));
@@ -181,6 +185,124 @@ graphkv_status run_score(const Dims &d, const Layout &l, const T *Q, const T *K,
     return launch_status();
 }
 
+// ---- step (I), tensor-core path (bf16) -----------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// Tensor map over K [batch][hkv][rows][128] bf16 with the caller's strides; boxes of 128 rows x 64
+// columns, 128-byte swizzle, zero fill past the last row.
+bool make_k_tensormap(CUtensorMap *tm, const void *K, const Dims &d, int rows)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t row_b = (cuuint64_t)d.ks[2] * 2;
+    cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows, (cuuint64_t)d.hkv, (cuuint64_t)d.batch};
+    cuuint64_t head_b = (cuuint64_t)d.ks[1] * 2, batch_b = (cuuint64_t)d.ks[0] * 2;
+    if (d.hkv == 1 || head_b == 0) head_b = row_b * (cuuint64_t)rows;
+    if (d.batch == 1 || batch_b == 0) batch_b = head_b * (cuuint64_t)d.hkv;
+    cuuint64_t strides[3] = {row_b, head_b, batch_b};
+    cuuint32_t box[4] = {64, (cuuint32_t)tc::kTileKeys, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(K), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int env_int(const char *name, int dflt)
+{
+    const char *v = getenv(name);
+    return v ? atoi(v) : dflt;
+}
+
+// Units per launch group: the group's keys should stay in L2 between the two sweeps.
+int units_per_group(const Dims &d)
+{
+    const double mb = (double)d.L * kHeadDim * 2 / 1.0e6;
+    int n = (int)(env_int("GRAPHKV_L2_GROUP_MB", 72) / mb);
+    if (n < 1) n = 1;
+    if (n > d.units) n = d.units;
+    return n;
+}
+
+template <typename Kern> bool set_smem(Kern k, size_t bytes)
+{
+    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
+graphkv_status run_score_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
+                            const __nv_bfloat16 *K, float *scores, void *ws, cudaStream_t st)
+{
+    CUtensorMap tmK;
+    if (!make_k_tensormap(&tmK, K, d, d.L)) return GRAPHKV_ERR_CUDA;
+    const int row_tiles = d.GW <= 128 ? 1 : 2;
+    const int rows_pad = 128 * row_tiles;
+    const int stages = row_tiles == 1 ? 5 : 4;
+    const size_t smem = tc::score_smem_bytes(rows_pad, stages);
+    static bool attr = false;
+    if (!attr) {
+        const size_t mx = tc::score_smem_bytes(256, 4) > tc::score_smem_bytes(128, 5)
+                              ? tc::score_smem_bytes(256, 4) : tc::score_smem_bytes(128, 5);
+        if (!set_smem(tc::score_stats_tc<1>, mx) || !set_smem(tc::score_stats_tc<2>, mx) ||
+            !set_smem(tc::score_emit_tc<1>, mx) || !set_smem(tc::score_emit_tc<2>, mx))
+            return GRAPHKV_ERR_CUDA;
+        attr = true;
+    }
+    float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
+    const int n_sms = 148;
+    const int tiles_stats = ceil_div(d.L, tc::kTileKeys), tiles_emit = ceil_div(d.N, tc::kTileKeys);
+    const int group = units_per_group(d);
+    for (int u0 = 0; u0 < d.units; u0 += group) {
+        const int nu = std::min(group, d.units - u0);
+        int chunks_s = std::max(1, std::min(n_sms / nu, tiles_stats));
+        chunks_s = std::min(chunks_s, l.max_parts / 2);
+        const int chunks_e = std::max(1, std::min(n_sms / nu, tiles_emit));
+        tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), a, at<int>(ws, l.status), u0, chunks_s,
+                           tiles_stats, 2 * chunks_s, stages};
+        tc::ScoreTcArgs ea = sa;
+        ea.chunks = chunks_e;
+        ea.n_tiles = tiles_emit;
+        if (row_tiles == 1) {
+            GKV_LAUNCH("score_stats_tc", st,
+                       (tc::score_stats_tc<1><<<dim3(chunks_s, nu), tc::kScoreThreads, smem, st>>>(tmK, sa)));
+            GKV_LAUNCH("score_emit_tc", st,
+                       (tc::score_emit_tc<1><<<dim3(chunks_e, nu), tc::kScoreThreads, smem, st>>>(tmK, ea)));
+        } else {
+            GKV_LAUNCH("score_stats_tc", st,
+                       (tc::score_stats_tc<2><<<dim3(chunks_s, nu), tc::kScoreThreads, smem, st>>>(tmK, sa)));
+            GKV_LAUNCH("score_emit_tc", st,
+                       (tc::score_emit_tc<2><<<dim3(chunks_e, nu), tc::kScoreThreads, smem, st>>>(tmK, ea)));
+        }
+    }
+    if (d.kp > 1)
+        GKV_LAUNCH("pool_max", st,
+                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a,
+                                                                                      scores)));
+    return launch_status();
+}
+
+inline graphkv_status run_score_any(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
+                                    const __nv_bfloat16 *K, float *scores, void *ws, cudaStream_t st)
+{
+    if (env_int("GRAPHKV_FORCE_SIMT", 0)) return run_score(d, l, Q, K, scores, ws, st);
+    return run_score_tc(d, l, Q, K, scores, ws, st);
+}
+
 // ---- steps (II)+(III) ------------------------------------------------------------------------
 template <typename T>
 graphkv_status run_propagate(const Dims &d, const Layout &l, const T *K, float *scores,
@@ -255,8 +377,8 @@ graphkv_status graphkv_score(const graphkv_params *params, const void *Qw, const
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (params->dtype == GRAPHKV_BF16)
-        return run_score(d, l, static_cast<const __nv_bfloat16 *>(Qw),
-                         static_cast<const __nv_bfloat16 *>(K), scores, workspace, st);
+        return run_score_any(d, l, static_cast<const __nv_bfloat16 *>(Qw),
+                             static_cast<const __nv_bfloat16 *>(K), scores, workspace, st);
     return run_score(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), scores,
                      workspace, st);
 }
@@ -315,8 +437,8 @@ graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, co
     float *s = scores_out ? scores_out : at<float>(workspace, l.s);
     const int elem = params->dtype == GRAPHKV_BF16 ? 2 : 4;
     if (params->dtype == GRAPHKV_BF16) {
-        rc = run_score(d, l, static_cast<const __nv_bfloat16 *>(Qw),
-                       static_cast<const __nv_bfloat16 *>(K), s, workspace, st);
+        rc = run_score_any(d, l, static_cast<const __nv_bfloat16 *>(Qw),
+                           static_cast<const __nv_bfloat16 *>(K), s, workspace, st);
         if (rc == GRAPHKV_OK)
             rc = run_propagate(d, l, static_cast<const __nv_bfloat16 *>(K), s, nullptr, workspace, st);
     } else {
