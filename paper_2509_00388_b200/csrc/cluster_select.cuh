@@ -1,0 +1,523 @@
+// Row-wise stages on thread-block clusters: one cluster of C CTAs owns the N scores of one
+// (sequence, KV head) unit, each CTA keeping a contiguous chunk of the row in shared memory.
+//
+//   pool_select_kernel   max pooling of the attention mass (step (I), last part) and the
+//                        source nodes of Eq. 2: top-k of the pooled scores.
+//   finish_kernel        the decay rounds of Eq. 5 / Algorithm 2 over the fixed neighbour lists,
+//                        the final k_l selection and the gather of the compact cache.
+//
+// Every exact top-k here is a most-significant-digit radix search over the order-preserving
+// uint32 image of the fp32 scores (digits of 11, 11 and 10 bits).  Per digit each CTA
+// histograms its chunk, the cluster reduces the histograms through distributed shared memory,
+// and every CTA locates the digit of the k-th largest value.  The kept indices come out in
+// ascending position; among equal values the lowest indices are kept.
+#pragma once
+
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace graphkv {
+namespace cs {
+
+namespace cg = cooperative_groups;
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kBins = 2048;
+constexpr int kMaxChunk = 32768;       // scores of a row one CTA keeps in shared memory
+constexpr int kMaxCluster = 8;
+constexpr int kMaxHalo = 64;           // (pool_kernel - 1) / 2 the pooling path handles
+constexpr int kMaxPerThread = kMaxChunk / kThreads;
+constexpr int kStage = 2048;           // neighbour-list entries staged in shared memory at a time
+constexpr int kMergeWarps = 8;         // warps of a CTA that merge candidate lists at a time
+constexpr int kSurvCap = 256;          // merged candidates one warp ranks in shared memory
+static_assert(kMergeWarps * kSurvCap * sizeof(Cand) <= 2 * kStage * 4, "survivors reuse the staging area");
+
+// Shared-memory carve-up common to both kernels (dynamic shared memory, 16-byte aligned).
+struct Smem {
+    uint32_t *hist;       // [kBins] this CTA's digit histogram
+    uint32_t *tot;        // [kBins] cluster-wide histogram (every CTA holds a copy)
+    uint32_t *wcnt;       // [2 * kWarps] per-warp counts
+    uint32_t *misc;       // [16] broadcast words and this CTA's published counts
+    int *st_idx;          // [kStage] staged neighbour positions, relative to the chunk
+    float *st_f;          // [kStage] their decay factors
+    float *vals;          // [halo + chunk + halo]
+};
+
+__host__ __device__ inline size_t smem_bytes(int chunk, int halo)
+{
+    return (size_t)(2 * kBins + 2 * kWarps + 16 + 2 * kStage) * 4 + (size_t)(chunk + 2 * halo + 8) * 4;
+}
+
+__device__ __forceinline__ Smem carve(uint8_t *raw, int halo)
+{
+    Smem s;
+    s.hist = reinterpret_cast<uint32_t *>(raw);
+    s.tot = s.hist + kBins;
+    s.wcnt = s.tot + kBins;
+    s.misc = s.wcnt + 2 * kWarps;
+    s.st_idx = reinterpret_cast<int *>(s.misc + 16);
+    s.st_f = reinterpret_cast<float *>(s.st_idx + kStage);
+    s.vals = s.st_f + kStage;
+    (void)halo;
+    return s;
+}
+
+// Result of the radix search: elements whose masked key exceeds `prefix` are kept, and of those
+// whose masked key equals it the `remaining` lowest indices.
+struct Threshold {
+    uint32_t prefix, mask, remaining;
+};
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// k-th largest of the cluster's row.  vals: this CTA's chunk (n_local elements, shared memory).
+// All CTAs of the cluster call this with the same k (1 <= k <= elements in the row) and return
+// the same Threshold.  Executes the same number of cluster barriers in every CTA.
+__device__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                 const float *vals, int n_local, uint32_t k)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    Threshold th{0u, 0u, k};
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const uint32_t nb = pass == 2 ? 1024u : 2048u;
+        for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0u;
+        __syncthreads();
+        for (int i0 = 0; i0 < n_local; i0 += kThreads) {
+            const int i = i0 + tid;
+            bool valid = i < n_local;
+            uint32_t bin = 0;
+            if (valid) {
+                const uint32_t u = float_to_key(vals[i]);
+                valid = (u & th.mask) == th.prefix;
+                bin = (u >> shift) & (nb - 1u);
+            }
+            // lanes sharing the first valid lane's digit are counted with one atomic (scores of a
+            // row often crowd into one digit); the others add for themselves
+            const unsigned vm = __ballot_sync(0xffffffffu, valid);
+            if (vm) {
+                const int leader = __ffs(vm) - 1;
+                const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
+                const bool same = valid && bin == lbin;
+                const unsigned sm = __ballot_sync(0xffffffffu, same);
+                if (lane == leader) atomicAdd(&s.hist[lbin], (uint32_t)__popc(sm));
+                else if (valid && !same) atomicAdd(&s.hist[bin], 1u);
+            }
+        }
+        __syncthreads();
+        const uint32_t *total = s.hist;
+        if (C > 1) {
+            cl.sync();                                   // every CTA's histogram is complete
+            const int slice = kBins / C;
+            if (tid < slice) {
+                const int bin = rank * slice + tid;
+                uint32_t sum = 0;
+                for (int p = 0; p < C; ++p) sum += cl.map_shared_rank(s.hist, p)[bin];
+                for (int p = 0; p < C; ++p) cl.map_shared_rank(s.tot, p)[bin] = sum;
+            }
+            cl.sync();                                   // every CTA's copy of the totals is complete
+            total = s.tot;
+        }
+        // walk the digits from the largest down: thread t owns digits nb-1-2t and nb-2-2t
+        uint32_t c0 = 0, c1 = 0;
+        if (2 * tid < (int)nb) {
+            c0 = total[nb - 1 - 2 * tid];
+            c1 = total[nb - 2 - 2 * tid];
+        }
+        uint32_t incl = warp_incl_scan(c0 + c1, lane);
+        if (lane == 31) s.wcnt[warp] = incl;
+        __syncthreads();
+        if (warp == 0) s.wcnt[lane] = warp_incl_scan(s.wcnt[lane], lane);
+        __syncthreads();
+        incl += warp == 0 ? 0u : s.wcnt[warp - 1];
+        const uint32_t before0 = incl - c0 - c1, before1 = before0 + c0;
+        if (before0 < th.remaining && before0 + c0 >= th.remaining) {
+            s.misc[0] = nb - 1 - 2 * tid;
+            s.misc[1] = th.remaining - before0;
+            s.misc[2] = c0;
+        } else if (before1 < th.remaining && before1 + c1 >= th.remaining) {
+            s.misc[0] = nb - 2 - 2 * tid;
+            s.misc[1] = th.remaining - before1;
+            s.misc[2] = c1;
+        }
+        __syncthreads();
+        th.prefix |= s.misc[0] << shift;
+        th.mask |= (nb - 1u) << shift;
+        th.remaining = s.misc[1];
+        const bool whole_class = s.misc[2] == th.remaining;
+        __syncthreads();
+        if (whole_class) break;       // every element of the threshold class is kept
+    }
+    return th;
+}
+
+// Ascending positions of the kept elements of the cluster's row -> out[0..k).  Returns nothing;
+// ends with the writes of this CTA issued (callers fence before another CTA reads them).
+// One cluster barrier.
+__device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                    const float *vals, int n_local, int base, Threshold th,
+                                    int *out)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // warp w owns the contiguous segment [w * seg, (w + 1) * seg) of the chunk
+    const int seg = ((n_local + kWarps - 1) / kWarps + 31) & ~31;
+    const int lo = min(warp * seg, n_local), hi = min(lo + seg, n_local);
+    uint32_t gt = 0, eq = 0;
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        const int i = i0 + lane;
+        uint32_t mk = 0;
+        const bool in = i < hi;
+        if (in) mk = float_to_key(vals[i]) & th.mask;
+        gt += __popc(__ballot_sync(0xffffffffu, in && mk > th.prefix));
+        eq += __popc(__ballot_sync(0xffffffffu, in && mk == th.prefix));
+    }
+    if (lane == 0) {
+        s.wcnt[warp] = gt;
+        s.wcnt[kWarps + warp] = eq;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t g = s.wcnt[lane], e = s.wcnt[kWarps + lane];
+        const uint32_t gi = warp_incl_scan(g, lane), ei = warp_incl_scan(e, lane);
+        s.wcnt[lane] = gi - g;                  // exclusive prefix over warps
+        s.wcnt[kWarps + lane] = ei - e;
+        if (lane == 31) {
+            s.misc[4] = gi;                     // this CTA's totals, read by the other ranks
+            s.misc[5] = ei;
+        }
+    }
+    __syncthreads();
+    uint32_t gt_before = s.wcnt[warp], eq_before = s.wcnt[kWarps + warp];
+    if (C > 1) {
+        cl.sync();
+        for (int p = 0; p < rank; ++p) {
+            const uint32_t *pm = cl.map_shared_rank(s.misc, p);
+            gt_before += pm[4];
+            eq_before += pm[5];
+        }
+    }
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        const int i = i0 + lane;
+        uint32_t mk = 0;
+        const bool in = i < hi;
+        if (in) mk = float_to_key(vals[i]) & th.mask;
+        const bool is_gt = in && mk > th.prefix, is_eq = in && mk == th.prefix;
+        const unsigned bg = __ballot_sync(0xffffffffu, is_gt), be = __ballot_sync(0xffffffffu, is_eq);
+        const unsigned below = (1u << lane) - 1u;
+        const uint32_t g = gt_before + __popc(bg & below), e = eq_before + __popc(be & below);
+        if (is_gt || (is_eq && e < th.remaining)) out[g + min(e, th.remaining)] = base + i;
+        gt_before += __popc(bg);
+        eq_before += __popc(be);
+    }
+}
+
+// Eq. 3 for one source: the m largest edges (cosine descending, position ascending) among the
+// candidate lists its key chunks wrote.  One warp; `surv` holds kSurvCap entries of shared memory.
+// The lists together hold every member of the top-m, and `hist` counts the listed edges per cosine
+// bin: the highest bin b with at least m listed edges in bins >= b bounds the m-th largest from
+// below, so only edges with e >= b / kCandBins need ranking.
+__device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chunks, int m,
+                                 Cand *surv, int *nbr_idx, float *nbr_e)
+{
+    const int lane = threadIdx.x & 31;
+    constexpr int kPer = kCandBins / 32;
+    // lane l holds bins [l * kPer, (l + 1) * kPer); walk down from the top bin
+    uint32_t h[kPer], mine = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        h[q] = __ldcg(hist + lane * kPer + q);
+        mine += h[q];
+    }
+    uint32_t above = 0;                       // listed edges in the lanes above this one
+    for (int l = 31; l > 0; --l) {
+        const uint32_t t = __shfl_sync(0xffffffffu, mine, l);
+        if (lane < l) above += t;
+    }
+    int bstar = -1;
+    uint32_t run = above;
+#pragma unroll
+    for (int q = kPer - 1; q >= 0; --q) {
+        run += h[q];
+        if (bstar < 0 && run >= (uint32_t)m) bstar = lane * kPer + q;
+    }
+    // the answer is the highest bin found by any lane
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bstar = max(bstar, __shfl_xor_sync(0xffffffffu, bstar, o));
+    const float bound = bstar <= 0 ? -1.0f : (float)bstar / (float)kCandBins;
+
+    const int slots = chunks * kCandCap;
+    int ns = 0;
+    for (int i0 = 0; i0 < slots; i0 += 128) {
+        unsigned long long raw[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * 32 + lane;
+            raw[q] = i < slots ? __ldcg(reinterpret_cast<const unsigned long long *>(cand + i)) : 0ull;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * 32 + lane;
+            const Cand cd{__uint_as_float(static_cast<uint32_t>(raw[q])), static_cast<int>(raw[q] >> 32)};
+            const bool keep = i < slots && cd.e >= bound;
+            const unsigned bm = __ballot_sync(0xffffffffu, keep);
+            const int pos = ns + __popc(bm & ((1u << lane) - 1u));
+            if (keep && pos < kSurvCap) surv[pos] = cd;
+            ns += __popc(bm);
+        }
+    }
+    if (ns > kSurvCap) {
+        // too many ties at the bound: exact m-th largest by bisection over the lists themselves
+        unsigned long long t64 = 0ull;
+        for (int bit = 63; bit >= 0; --bit) {
+            const unsigned long long cut = t64 | (1ull << bit);
+            int n = 0;
+            for (int i = lane; i < slots; i += 32) {
+                const unsigned long long raw = __ldcg(reinterpret_cast<const unsigned long long *>(cand + i));
+                const float e = __uint_as_float(static_cast<uint32_t>(raw));
+                n += e >= -1.0f && edge_key(e, static_cast<int>(raw >> 32)) >= cut;
+            }
+            n = __reduce_add_sync(0xffffffffu, n);
+            if (n >= m) t64 = cut;
+        }
+        ns = 0;
+        for (int i0 = 0; i0 < slots; i0 += 32) {
+            const int i = i0 + lane;
+            bool keep = false;
+            Cand cd{0.f, 0};
+            if (i < slots) {
+                const unsigned long long raw = __ldcg(reinterpret_cast<const unsigned long long *>(cand + i));
+                cd.e = __uint_as_float(static_cast<uint32_t>(raw));
+                cd.j = static_cast<int>(raw >> 32);
+                keep = cd.e >= -1.0f && edge_key(cd.e, cd.j) >= t64;
+            }
+            const unsigned bm = __ballot_sync(0xffffffffu, keep);
+            const int pos = ns + __popc(bm & ((1u << lane) - 1u));
+            if (keep && pos < kSurvCap) surv[pos] = cd;
+            ns += __popc(bm);
+        }
+    }
+    __syncwarp();
+    // rank by counting: all keys are distinct (distinct positions)
+    for (int i = lane; i < ns; i += 32) {
+        const Cand me = surv[i];
+        const unsigned long long k = edge_key(me.e, me.j);
+        int rank = 0;
+        for (int t = 0; t < ns; ++t) rank += edge_key(surv[t].e, surv[t].j) > k;
+        if (rank < m) {
+            nbr_idx[rank] = me.j;
+            nbr_e[rank] = me.e;
+        }
+    }
+    __syncwarp();
+}
+
+struct PoolSelectArgs {
+    Dims d;
+    int C, chunk, halo;
+    int unit0;
+    const float *a;        // [units][N] attention mass before pooling, or nullptr: no pooling
+    float *s;              // [units][N] scores: written when pooling, read otherwise
+    int k;                 // sources to pick (0: none)
+    int *src_out;          // [units][k] ascending positions
+    uint32_t *zero;        // optional: [units][zero_words] words this launch clears for later kernels
+    int zero_words;
+};
+
+// grid = units * C CTAs in clusters of C; block kThreads.
+__global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs a)
+{
+    extern __shared__ __align__(16) uint8_t cs_smem[];
+    cg::cluster_group cl = cg::this_cluster();
+    const int C = a.C, rank = C > 1 ? (int)cl.block_rank() : 0;
+    const int unit = a.unit0 + blockIdx.x / C;
+    const Smem s = carve(cs_smem, a.halo);
+    const int N = a.d.N, tid = threadIdx.x;
+    const int base = rank * a.chunk;
+    const int n_local = max(0, min(a.chunk, N - base));
+    float *vals = s.vals + a.halo;
+    float *row_s = a.s + (long long)unit * N;
+    if (a.zero)
+        for (int i = rank * kThreads + tid; i < a.zero_words; i += C * kThreads)
+            a.zero[(long long)unit * a.zero_words + i] = 0u;
+    if (a.a) {
+        const float *row_a = a.a + (long long)unit * N;
+        const int half = a.halo;
+        for (int i = tid - half; i < n_local + half; i += kThreads) {
+            const int j = base + i;
+            vals[i] = (n_local > 0 && j >= 0 && j < N) ? row_a[j] : -INFINITY;
+        }
+        __syncthreads();
+        float pooled[kMaxPerThread];
+#pragma unroll
+        for (int q = 0; q < kMaxPerThread; ++q) {
+            const int i = q * kThreads + tid;
+            if (i < n_local) {
+                float best = vals[i - half];
+                for (int t = 1 - half; t <= half; ++t) best = fmaxf(best, vals[i + t]);
+                pooled[q] = best;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kMaxPerThread; ++q) {
+            const int i = q * kThreads + tid;
+            if (i < n_local) {
+                vals[i] = pooled[q];
+                row_s[base + i] = pooled[q];
+            }
+        }
+    } else {
+        for (int i = tid; i < n_local; i += kThreads) vals[i] = row_s[base + i];
+    }
+    __syncthreads();
+    if (a.k > 0) {
+        const Threshold th = cluster_kth(cl, C, rank, s, vals, n_local, (uint32_t)a.k);
+        cluster_emit_sorted(cl, C, rank, s, vals, n_local, base, th,
+                            a.src_out + (long long)unit * a.k);
+    }
+    if (C > 1) cl.sync();      // no CTA leaves while its shared memory may still be read
+}
+
+struct FinishArgs {
+    Dims d;
+    int C, chunk;
+    int unit0;
+    float *s;                  // [units][N] scores (decayed in place when has_graph)
+    int *nbr_idx;              // [units][K_src][m] neighbour lists (has_graph); written when merging
+    float *nbr_e;              // [units][K_src][m] their cosines
+    int has_graph;             // apply the decay rounds
+    int merge;                 // build the neighbour lists from the per-chunk candidate lists first
+    const Cand *cand;          // [units][K_src][cand_chunks][kCandCap]
+    const uint32_t *cand_hist; // [units][K_src][kCandBins]
+    int cand_chunks;
+    int do_select;             // pick the budget and gather
+    int *idx_out;              // [units][B]
+    int elem_bytes;
+    const unsigned char *K, *V;
+    unsigned char *K_out, *V_out;
+};
+
+// grid = units * C CTAs in clusters of C; block kThreads.
+__global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
+{
+    extern __shared__ __align__(16) uint8_t cs_smem[];
+    cg::cluster_group cl = cg::this_cluster();
+    const Dims &d = a.d;
+    const int C = a.C, rank = C > 1 ? (int)cl.block_rank() : 0;
+    const int unit = a.unit0 + blockIdx.x / C;
+    const Smem s = carve(cs_smem, 0);
+    const int N = d.N, tid = threadIdx.x;
+    const int base = rank * a.chunk;
+    const int n_local = max(0, min(a.chunk, N - base));
+    float *vals = s.vals;
+    float *row_s = a.s + (long long)unit * N;
+    for (int i = tid; i < n_local; i += kThreads) vals[i] = row_s[base + i];
+    __syncthreads();
+
+    if (a.has_graph && a.merge) {
+        // Eq. 3: warp w of rank r merges sources (w + kMergeWarps * t) * C + r
+        const int warp = tid >> 5;
+        if (warp < kMergeWarps) {
+            Cand *surv = reinterpret_cast<Cand *>(s.st_idx) + warp * kSurvCap;
+            for (int src = warp * C + rank; src < d.K_src; src += kMergeWarps * C) {
+                const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
+                merge_neighbours(a.cand + slot * kCandCap,
+                                 a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
+                                 a.cand_chunks, d.m, surv,
+                                 a.nbr_idx + ((long long)unit * d.K_src + src) * d.m,
+                                 a.nbr_e + ((long long)unit * d.K_src + src) * d.m);
+            }
+        }
+        __threadfence();
+        if (C > 1) cl.sync(); else __syncthreads();
+    }
+
+    if (a.has_graph) {
+        // Eq. 5 over the fixed graph: source after source (a source's neighbours are distinct, so
+        // one source is applied by parallel threads), the T rounds folded into a power.
+        const int *ni = a.nbr_idx + (long long)unit * d.K_src * d.m;
+        const float *ne = a.nbr_e + (long long)unit * d.K_src * d.m;
+        const int per = d.m <= kStage ? kStage / d.m : 0;      // sources staged together
+        if (per > 0) {
+            for (int src0 = 0; src0 < d.K_src; src0 += per) {
+                const int ns = min(per, d.K_src - src0);
+                for (int i = tid; i < ns * d.m; i += kThreads) {
+                    const float f = 1.0f - d.lambda * fmaxf(__ldcg(ne + src0 * d.m + i), 0.f);
+                    float pw = f;
+                    for (int t = 1; t < d.T; ++t) pw *= f;
+                    s.st_idx[i] = __ldcg(ni + src0 * d.m + i) - base;
+                    s.st_f[i] = pw;
+                }
+                __syncthreads();
+                for (int q = 0; q < ns; ++q) {
+                    for (int u = tid; u < d.m; u += kThreads) {
+                        const int j = s.st_idx[q * d.m + u];
+                        if (j >= 0 && j < n_local) vals[j] *= s.st_f[q * d.m + u];
+                    }
+                    __syncthreads();
+                }
+            }
+        } else {
+            for (int src = 0; src < d.K_src; ++src) {
+                for (int u = tid; u < d.m; u += kThreads) {
+                    const int j = ni[src * d.m + u] - base;
+                    if (j >= 0 && j < n_local) {
+                        const float f = 1.0f - d.lambda * fmaxf(ne[src * d.m + u], 0.f);
+                        float pw = f;
+                        for (int t = 1; t < d.T; ++t) pw *= f;
+                        vals[j] *= pw;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        for (int i = tid; i < n_local; i += kThreads) row_s[base + i] = vals[i];
+    }
+
+    if (a.do_select) {
+        int *idx = a.idx_out + (long long)unit * d.B;
+        const Threshold th = cluster_kth(cl, C, rank, s, vals, n_local, (uint32_t)d.B);
+        cluster_emit_sorted(cl, C, rank, s, vals, n_local, base, th, idx);
+        __threadfence();
+        if (C > 1) cl.sync(); else __syncthreads();
+        // gather: the cluster's threads share the 16-byte pieces of the B + W output rows
+        if (a.K || a.V) {
+            const int vec_per_row = kHeadDim * a.elem_bytes / 16;
+            const int rows_out = d.B + d.W;
+            const long long row_bytes = (long long)kHeadDim * a.elem_bytes;
+            const int b = unit / d.hkv, h = unit % d.hkv;
+            const long long total = (long long)rows_out * vec_per_row;
+            for (long long p = (long long)rank * kThreads + tid; p < total; p += (long long)C * kThreads) {
+                const int c = (int)(p % vec_per_row);
+                const int t = (int)(p / vec_per_row);
+                const int src_row = t < d.B ? __ldcg(idx + t) : N + (t - d.B);
+                const long long dst = ((long long)unit * rows_out + t) * row_bytes + c * 16;
+                if (a.K) {
+                    const long long off = (b * d.ks[0] + h * d.ks[1] + src_row * d.ks[2]) * a.elem_bytes;
+                    *reinterpret_cast<uint4 *>(a.K_out + dst) =
+                        *reinterpret_cast<const uint4 *>(a.K + off + c * 16);
+                }
+                if (a.V) {
+                    const long long off = (b * d.vs[0] + h * d.vs[1] + src_row * d.vs[2]) * a.elem_bytes;
+                    *reinterpret_cast<uint4 *>(a.V_out + dst) =
+                        *reinterpret_cast<const uint4 *>(a.V + off + c * 16);
+                }
+            }
+        }
+    }
+    if (C > 1) cl.sync();      // no CTA leaves while its shared memory may still be read
+}
+
+}  // namespace cs
+}  // namespace graphkv

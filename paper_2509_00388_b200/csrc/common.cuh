@@ -54,6 +54,29 @@ __device__ __forceinline__ uint32_t float_to_key(float x)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// A listed edge: cosine and the position of the key it leads to.
+struct Cand {
+    float e;
+    int j;
+};
+constexpr int kCandCap = 64;            // candidate slots per (source, key chunk)
+constexpr int kCandBins = 256;          // cosine bins of the per-source candidate histogram
+constexpr float kCandEmpty = -2.0f;     // cosine stored in an unused slot (valid cosines are >= -1)
+
+// Bin of a cosine: floor(e * kCandBins) clamped to [0, kCandBins); e >= b / kCandBins exactly when
+// its bin is >= b (the scaling is exact in binary floating point).
+__device__ __forceinline__ int cand_bin(float e)
+{
+    return min(max(static_cast<int>(floorf(e * kCandBins)), 0), kCandBins - 1);
+}
+
+// Order-preserving 64-bit image of an edge: larger cosine first, then lower position.
+__device__ __forceinline__ unsigned long long edge_key(float e, int j)
+{
+    return (static_cast<unsigned long long>(float_to_key(e)) << 32) |
+           static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(j));
+}
+
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll

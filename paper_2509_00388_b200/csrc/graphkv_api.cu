@@ -7,12 +7,14 @@
 #include <mutex>
 #include <vector>
 
+#include "cluster_select.cuh"
 #include "common.cuh"
 #include "gather.cuh"
 #include "propagate_simt.cuh"
 #include "score_simt.cuh"
 #include "score_tc.cuh"
 #include "select.cuh"
+#include "sim_tc.cuh"
 
 using namespace graphkv;
 
@@ -31,6 +33,8 @@ struct Layout {
     size_t sims;        // edges of the sources [units][K_src][N]
     size_t nbr_idx;     // neighbourhoods [units][K_src][m]
     size_t nbr_e;
+    size_t cand;        // per-chunk neighbour candidates [units][K_src][sim_chunks][kCandCap]
+    size_t cand_hist;   // [units][K_src][kCandBins]
     size_t total;
     int n_stat_chunks;  // key chunks of the SIMT statistics sweep
     int max_parts;      // partial statistics per row the region can hold
@@ -75,6 +79,45 @@ graphkv_status resolve(const graphkv_params *p, Dims *d)
     return GRAPHKV_OK;
 }
 
+int env_int(const char *name, int dflt)
+{
+    const char *v = getenv(name);
+    return v ? atoi(v) : dflt;
+}
+
+// Units per launch group: the group's keys should stay in L2 between the sweeps.
+int units_per_group(const Dims &d)
+{
+    const double mb = (double)d.L * kHeadDim * 2 / 1.0e6;
+    int n = (int)(env_int("GRAPHKV_L2_GROUP_MB", 72) / mb);
+    if (n < 1) n = 1;
+    if (n > d.units) n = d.units;
+    return n;
+}
+
+// Tensor-core similarity sweep: usable for bf16 keys, up to 64 sources and 32 neighbours.
+struct SimPlan {
+    bool ok;
+    int NP;         // source count padded to 16, 32 or 64
+    int chunks;     // CTAs (key chunks) per unit
+    int n_tiles;    // 128-key tiles per unit
+    int stages;
+};
+
+SimPlan sim_plan(const Dims &d, bool bf16)
+{
+    SimPlan p{false, 16, 1, ceil_div(d.N, tc::kTileKeys), 5};
+    if (!bf16 || d.K_src < 1 || d.K_src > 64 || d.m < 1 || d.m > tc::kSimMaxNeighbors) return p;
+    if (env_int("GRAPHKV_FORCE_SIMT", 0)) return p;
+    p.NP = d.K_src <= 16 ? 16 : (d.K_src <= 32 ? 32 : 64);
+    p.stages = p.NP == 64 ? 4 : 5;
+    const int cap = 512 / p.NP;
+    const int group = units_per_group(d);
+    p.chunks = std::max(ceil_div(p.n_tiles, cap), std::max(1, std::min(148 / group, p.n_tiles)));
+    p.ok = true;
+    return p;
+}
+
 Layout layout_of(const Dims &d)
 {
     Layout l;
@@ -91,6 +134,10 @@ Layout layout_of(const Dims &d)
     l.sims = take((size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * d.N * sizeof(float));
     l.nbr_idx = take(pairs * sizeof(int));
     l.nbr_e = take(pairs * sizeof(float));
+    const SimPlan sp = sim_plan(d, true);
+    const size_t slots = sp.ok ? (size_t)d.units * d.K_src * sp.chunks : 1;
+    l.cand = take(slots * kCandCap * sizeof(Cand));
+    l.cand_hist = take((size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * kCandBins * sizeof(uint32_t));
     l.total = off;
     return l;
 }
@@ -156,12 +203,12 @@ template <typename T> inline T *at(void *ws, size_t off)
 }
 
 // ---- step (I) ------------------------------------------------------------------------------
+// Attention mass before pooling, a [units][N], SIMT path (any dtype).
 template <typename T>
-graphkv_status run_score(const Dims &d, const Layout &l, const T *Q, const T *K, float *scores,
-                         void *ws, cudaStream_t st)
+graphkv_status run_mass_simt(const Dims &d, const Layout &l, const T *Q, const T *K, float *a,
+                             void *ws, cudaStream_t st)
 {
     float *part = at<float>(ws, l.part);
-    float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
     const int threads = ceil_div(d.GW, 32) * 32;
     GKV_LAUNCH("score_stats_simt", st,
                (score_stats_simt<T><<<dim3(l.n_stat_chunks, d.units), threads, 0, st>>>(
@@ -178,10 +225,6 @@ graphkv_status run_score(const Dims &d, const Layout &l, const T *Q, const T *K,
     GKV_LAUNCH("score_emit_simt", st,
                (score_emit_simt<T><<<dim3(ceil_div(d.N, kEmitChunk), d.units), kEmitThreads, smem,
                                      st>>>(d, Q, K, part, l.n_stat_chunks, a)));
-    if (d.kp > 1)
-        GKV_LAUNCH("pool_max", st,
-                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a,
-                                                                                      scores)));
     return launch_status();
 }
 
@@ -224,29 +267,14 @@ bool make_k_tensormap(CUtensorMap *tm, const void *K, const Dims &d, int rows)
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int env_int(const char *name, int dflt)
-{
-    const char *v = getenv(name);
-    return v ? atoi(v) : dflt;
-}
-
-// Units per launch group: the group's keys should stay in L2 between the two sweeps.
-int units_per_group(const Dims &d)
-{
-    const double mb = (double)d.L * kHeadDim * 2 / 1.0e6;
-    int n = (int)(env_int("GRAPHKV_L2_GROUP_MB", 72) / mb);
-    if (n < 1) n = 1;
-    if (n > d.units) n = d.units;
-    return n;
-}
-
 template <typename Kern> bool set_smem(Kern k, size_t bytes)
 {
     return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
 }
 
-graphkv_status run_score_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
-                            const __nv_bfloat16 *K, float *scores, void *ws, cudaStream_t st)
+// Attention mass before pooling, a [units][N], tensor-core path (bf16).
+graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
+                           const __nv_bfloat16 *K, float *a, void *ws, cudaStream_t st)
 {
     CUtensorMap tmK;
     if (!make_k_tensormap(&tmK, K, d, d.L)) return GRAPHKV_ERR_CUDA;
@@ -263,7 +291,6 @@ graphkv_status run_score_tc(const Dims &d, const Layout &l, const __nv_bfloat16 
             return GRAPHKV_ERR_CUDA;
         attr = true;
     }
-    float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
     const int n_sms = 148;
     const int tiles_stats = ceil_div(d.L, tc::kTileKeys), tiles_emit = ceil_div(d.N, tc::kTileKeys);
     const int group = units_per_group(d);
@@ -289,30 +316,134 @@ graphkv_status run_score_tc(const Dims &d, const Layout &l, const __nv_bfloat16 
                        (tc::score_emit_tc<2><<<dim3(chunks_e, nu), tc::kScoreThreads, smem, st>>>(tmK, ea)));
         }
     }
-    if (d.kp > 1)
-        GKV_LAUNCH("pool_max", st,
-                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a,
-                                                                                      scores)));
     return launch_status();
 }
 
-inline graphkv_status run_score_any(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
-                                    const __nv_bfloat16 *K, float *scores, void *ws, cudaStream_t st)
+inline graphkv_status run_mass(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
+                               const __nv_bfloat16 *K, float *a, void *ws, cudaStream_t st)
 {
-    if (env_int("GRAPHKV_FORCE_SIMT", 0)) return run_score(d, l, Q, K, scores, ws, st);
-    return run_score_tc(d, l, Q, K, scores, ws, st);
+    if (env_int("GRAPHKV_FORCE_SIMT", 0)) return run_mass_simt(d, l, Q, K, a, ws, st);
+    return run_mass_tc(d, l, Q, K, a, ws, st);
+}
+inline graphkv_status run_mass(const Dims &d, const Layout &l, const float *Q, const float *K,
+                               float *a, void *ws, cudaStream_t st)
+{
+    return run_mass_simt(d, l, Q, K, a, ws, st);
 }
 
-// ---- steps (II)+(III) ------------------------------------------------------------------------
-template <typename T>
-graphkv_status run_propagate(const Dims &d, const Layout &l, const T *K, float *scores,
-                             int *src_out, void *ws, cudaStream_t st)
+// ---- row-wise stages on clusters -------------------------------------------------------------
+struct ClusterPlan {
+    bool ok;            // the row fits the cluster kernels
+    int C, chunk, halo;
+};
+
+ClusterPlan cluster_plan(const Dims &d)
 {
-    if (d.K_src == 0) return GRAPHKV_OK;
-    int *src = src_out ? src_out : at<int>(ws, l.src);
-    SelectArgs sa{scores, d.N, d.N, d.K_src, nullptr, src, nullptr};
-    GKV_LAUNCH("select_sources", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
-    if (d.T == 0 || d.m == 0) return launch_status();
+    ClusterPlan p{false, 1, 0, (d.kp - 1) / 2};
+    if (env_int("GRAPHKV_NO_CLUSTER", 0)) return p;
+    while (p.C < cs::kMaxCluster && ceil_div(d.N, p.C) > 4096) p.C *= 2;
+    p.chunk = (ceil_div(d.N, p.C) + 31) & ~31;
+    p.ok = p.chunk <= cs::kMaxChunk && p.halo <= cs::kMaxHalo;
+    return p;
+}
+
+template <typename Kern, typename Args>
+graphkv_status launch_cluster(const char *name, Kern kern, const Args &args, int clusters, int C,
+                              size_t smem, cudaStream_t st)
+{
+    static std::once_flag once;
+    static bool attr_ok = true;
+    std::call_once(once, [] {
+        const size_t mx = cs::smem_bytes(cs::kMaxChunk, cs::kMaxHalo);
+        attr_ok = set_smem(cs::pool_select_kernel, mx) && set_smem(cs::finish_kernel, mx);
+    });
+    if (!attr_ok) return GRAPHKV_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(clusters * C);
+    cfg.blockDim = dim3(cs::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    GKV_LAUNCH(name, st, (e = cudaLaunchKernelEx(&cfg, kern, args)));
+    if (e != cudaSuccess) {
+        if (getenv("GRAPHKV_LOG")) fprintf(stderr, "graphkv: %s: %s\n", name, cudaGetErrorString(e));
+        return GRAPHKV_ERR_CUDA;
+    }
+    return GRAPHKV_OK;
+}
+
+// Pooling of a -> s (when a != nullptr) and the k source nodes of Eq. 2 (when k > 0).
+// `zero` (optional): zero_words words per unit cleared on the way, for the kernels that follow.
+graphkv_status run_pool_sources(const Dims &d, const float *a, float *s, int k, int *src,
+                                uint32_t *zero, int zero_words, cudaStream_t st)
+{
+    if (!a && k == 0) return GRAPHKV_OK;
+    const ClusterPlan cp = cluster_plan(d);
+    if (cp.ok) {
+        cs::PoolSelectArgs pa{d, cp.C, cp.chunk, a ? cp.halo : 0, 0, a, s, k, src, zero, zero_words};
+        return launch_cluster(a ? (k ? "pool_select_sources" : "pool_max") : "select_sources",
+                              cs::pool_select_kernel, pa, d.units, cp.C,
+                              cs::smem_bytes(cp.chunk, pa.halo), st);
+    }
+    if (zero && cudaMemsetAsync(zero, 0, (size_t)d.units * zero_words * 4, st) != cudaSuccess)
+        return GRAPHKV_ERR_CUDA;
+    if (a)
+        GKV_LAUNCH("pool_max", st,
+                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a, s)));
+    if (k > 0) {
+        SelectArgs sa{s, d.N, d.N, k, nullptr, src, nullptr};
+        GKV_LAUNCH("select_sources", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
+    }
+    return launch_status();
+}
+
+// ---- steps (II)+(III): the graph ------------------------------------------------------------------
+inline bool graph_active(const Dims &d) { return d.K_src > 0 && d.T > 0 && d.m > 0; }
+
+// Edges of the sources (Eq. 1) and their top-m neighbourhoods (Eq. 3) -> neighbour lists in the
+// workspace.  `src` holds the sources in ascending position.
+template <typename T>
+graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *src, void *ws,
+                         cudaStream_t st)
+{
+    const SimPlan sp = sim_plan(d, sizeof(T) == 2);
+    if (sp.ok) {
+        CUtensorMap tmK;
+        if (!make_k_tensormap(&tmK, K, d, d.L)) return GRAPHKV_ERR_CUDA;
+        static std::once_flag once;
+        static bool attr_ok = true;
+        std::call_once(once, [] {
+            attr_ok = set_smem(tc::similarity_tc<16>, tc::sim_smem_bytes<16>(5)) &&
+                      set_smem(tc::similarity_tc<32>, tc::sim_smem_bytes<32>(5)) &&
+                      set_smem(tc::similarity_tc<64>, tc::sim_smem_bytes<64>(4));
+        });
+        if (!attr_ok) return GRAPHKV_ERR_CUDA;
+        const int group = units_per_group(d);
+        for (int u0 = 0; u0 < d.units; u0 += group) {
+            const int nu = std::min(group, d.units - u0);
+            tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(K), src, at<Cand>(ws, l.cand),
+                             at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
+                             sp.n_tiles, sp.stages};
+            const dim3 grid(sp.chunks, nu);
+            if (sp.NP == 16)
+                GKV_LAUNCH("similarity_tc", st,
+                           (tc::similarity_tc<16><<<grid, tc::kSimThreads, tc::sim_smem_bytes<16>(sp.stages), st>>>(tmK, sa)));
+            else if (sp.NP == 32)
+                GKV_LAUNCH("similarity_tc", st,
+                           (tc::similarity_tc<32><<<grid, tc::kSimThreads, tc::sim_smem_bytes<32>(sp.stages), st>>>(tmK, sa)));
+            else
+                GKV_LAUNCH("similarity_tc", st,
+                           (tc::similarity_tc<64><<<grid, tc::kSimThreads, tc::sim_smem_bytes<64>(sp.stages), st>>>(tmK, sa)));
+        }
+        return launch_status();
+    }
     float *sims = at<float>(ws, l.sims);
     GKV_LAUNCH("similarity_simt", st,
                (similarity_simt<T><<<dim3(ceil_div(d.N, kSimChunk), d.units), kSimThreads, 0, st>>>(
@@ -320,30 +451,91 @@ graphkv_status run_propagate(const Dims &d, const Layout &l, const T *K, float *
     SelectArgs na{sims, d.N, d.N, d.m, src, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e)};
     GKV_LAUNCH("select_neighbors", st,
                (topk_select_kernel<<<d.units * d.K_src, kSelectThreads, 0, st>>>(na)));
-    GKV_LAUNCH("decay_rounds", st,
-               (decay_rounds_kernel<<<d.units, 256, 0, st>>>(d, at<int>(ws, l.nbr_idx),
-                                                             at<float>(ws, l.nbr_e), scores)));
     return launch_status();
 }
 
-// ---- step (IV) ---------------------------------------------------------------------------------
-graphkv_status run_select_gather(const Dims &d, int elem_bytes, const float *scores, const void *K,
-                                 const void *V, void *K_out, void *V_out, int *idx_out,
-                                 cudaStream_t st)
+// Decay rounds (when has_graph) on s in place, then (when do_select) the budget selection and
+// the gather of the compact cache.
+graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, float *s, bool has_graph,
+                          bool merge, bool do_select, const void *K, const void *V, void *K_out, void *V_out,
+                          int *idx_out, void *ws, cudaStream_t st)
 {
-    SelectArgs sa{scores, d.N, d.N, d.B, nullptr, idx_out, nullptr};
-    GKV_LAUNCH("select_budget", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
-    if (K || V) {
-        const long long total = (long long)d.units * (d.B + d.W) * (kHeadDim * elem_bytes / 16);
-        const int blocks = (int)std::min<long long>((total + kGatherThreads - 1) / kGatherThreads,
-                                                    148LL * 16);
-        GKV_LAUNCH("gather_rows", st,
-                   (gather_rows_kernel<<<blocks, kGatherThreads, 0, st>>>(
-                       d, elem_bytes, static_cast<const unsigned char *>(K),
-                       static_cast<const unsigned char *>(V), idx_out,
-                       static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out))));
+    if (!has_graph && !do_select) return GRAPHKV_OK;
+    const ClusterPlan cp = cluster_plan(d);
+    if (cp.ok) {
+        cs::FinishArgs fa{d, cp.C, cp.chunk, 0, s, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e),
+                          has_graph ? 1 : 0, has_graph && merge ? 1 : 0, at<Cand>(ws, l.cand),
+                          at<uint32_t>(ws, l.cand_hist), sim_plan(d, true).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
+                          static_cast<const unsigned char *>(K), static_cast<const unsigned char *>(V),
+                          static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out)};
+        const char *name = has_graph ? (do_select ? "decay_select_gather" : "decay_rounds") : "select_gather";
+        return launch_cluster(name, cs::finish_kernel, fa, d.units, cp.C, cs::smem_bytes(cp.chunk, 0), st);
+    }
+    if (has_graph)
+        GKV_LAUNCH("decay_rounds", st,
+                   (decay_rounds_kernel<<<d.units, 256, 0, st>>>(d, at<int>(ws, l.nbr_idx),
+                                                                 at<float>(ws, l.nbr_e), s)));
+    if (do_select) {
+        SelectArgs sa{s, d.N, d.N, d.B, nullptr, idx_out, nullptr};
+        GKV_LAUNCH("select_budget", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
+        if (K || V) {
+            const long long total = (long long)d.units * (d.B + d.W) * (kHeadDim * elem_bytes / 16);
+            const int blocks = (int)std::min<long long>((total + kGatherThreads - 1) / kGatherThreads,
+                                                        148LL * 16);
+            GKV_LAUNCH("gather_rows", st,
+                       (gather_rows_kernel<<<blocks, kGatherThreads, 0, st>>>(
+                           d, elem_bytes, static_cast<const unsigned char *>(K),
+                           static_cast<const unsigned char *>(V), idx_out,
+                           static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out))));
+        }
     }
     return launch_status();
+}
+
+// ---- the calls, typed ---------------------------------------------------------------------------
+template <typename T>
+graphkv_status do_score(const Dims &d, const Layout &l, const T *Q, const T *K, float *scores,
+                        void *ws, cudaStream_t st)
+{
+    float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
+    graphkv_status rc = run_mass(d, l, Q, K, a, ws, st);
+    if (rc != GRAPHKV_OK || d.kp == 1) return rc;
+    return run_pool_sources(d, a, scores, 0, nullptr, nullptr, 0, st);
+}
+
+template <typename T>
+graphkv_status do_propagate(const Dims &d, const Layout &l, const T *K, float *scores, int *src_out,
+                            void *ws, cudaStream_t st)
+{
+    if (d.K_src == 0) return GRAPHKV_OK;
+    int *src = src_out ? src_out : at<int>(ws, l.src);
+    const bool tc_graph = graph_active(d) && sim_plan(d, sizeof(T) == 2).ok;
+    graphkv_status rc = run_pool_sources(d, nullptr, scores, d.K_src, src,
+                                         tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr,
+                                         d.K_src * kCandBins, st);
+    if (rc != GRAPHKV_OK || !graph_active(d)) return rc;
+    if ((rc = run_graph(d, l, K, src, ws, st)) != GRAPHKV_OK) return rc;
+    return run_finish(d, l, (int)sizeof(T), scores, true, sim_plan(d, sizeof(T) == 2).ok, false,
+                      nullptr, nullptr, nullptr, nullptr, nullptr, ws, st);
+}
+
+template <typename T>
+graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *K, const void *V,
+                           void *K_out, void *V_out, int *idx_out, float *s, void *ws,
+                           cudaStream_t st)
+{
+    const bool graph = graph_active(d);
+    float *a = d.kp > 1 ? at<float>(ws, l.a) : s;
+    graphkv_status rc = run_mass(d, l, Q, K, a, ws, st);
+    if (rc != GRAPHKV_OK) return rc;
+    int *src = at<int>(ws, l.src);
+    const bool tc_graph = graph && sim_plan(d, sizeof(T) == 2).ok;
+    rc = run_pool_sources(d, d.kp > 1 ? a : nullptr, s, graph ? d.K_src : 0, src,
+                          tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr, d.K_src * kCandBins, st);
+    if (rc != GRAPHKV_OK) return rc;
+    if (graph && (rc = run_graph(d, l, K, src, ws, st)) != GRAPHKV_OK) return rc;
+    return run_finish(d, l, (int)sizeof(T), s, graph, sim_plan(d, sizeof(T) == 2).ok, true, K, V,
+                      K_out, V_out, idx_out, ws, st);
 }
 
 }  // namespace
@@ -377,10 +569,10 @@ graphkv_status graphkv_score(const graphkv_params *params, const void *Qw, const
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (params->dtype == GRAPHKV_BF16)
-        return run_score_any(d, l, static_cast<const __nv_bfloat16 *>(Qw),
-                             static_cast<const __nv_bfloat16 *>(K), scores, workspace, st);
-    return run_score(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), scores,
-                     workspace, st);
+        return do_score(d, l, static_cast<const __nv_bfloat16 *>(Qw),
+                        static_cast<const __nv_bfloat16 *>(K), scores, workspace, st);
+    return do_score(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), scores,
+                    workspace, st);
 }
 
 graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, float *scores,
@@ -395,9 +587,9 @@ graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, fl
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (params->dtype == GRAPHKV_BF16)
-        return run_propagate(d, l, static_cast<const __nv_bfloat16 *>(K), scores, src_idx_out,
-                             workspace, st);
-    return run_propagate(d, l, static_cast<const float *>(K), scores, src_idx_out, workspace, st);
+        return do_propagate(d, l, static_cast<const __nv_bfloat16 *>(K), scores, src_idx_out,
+                            workspace, st);
+    return do_propagate(d, l, static_cast<const float *>(K), scores, src_idx_out, workspace, st);
 }
 
 graphkv_status graphkv_select_gather(const graphkv_params *params, const float *scores,
@@ -416,8 +608,8 @@ graphkv_status graphkv_select_gather(const graphkv_params *params, const float *
     const Layout l = layout_of(d);
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     const int elem = params->dtype == GRAPHKV_BF16 ? 2 : 4;
-    return run_select_gather(d, elem, scores, K, V, K_out, V_out, idx_out,
-                             static_cast<cudaStream_t>(stream));
+    return run_finish(d, l, elem, const_cast<float *>(scores), false, false, true, K, V, K_out, V_out,
+                      idx_out, workspace, static_cast<cudaStream_t>(stream));
 }
 
 graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, const void *K,
@@ -435,20 +627,12 @@ graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, co
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float *s = scores_out ? scores_out : at<float>(workspace, l.s);
-    const int elem = params->dtype == GRAPHKV_BF16 ? 2 : 4;
-    if (params->dtype == GRAPHKV_BF16) {
-        rc = run_score_any(d, l, static_cast<const __nv_bfloat16 *>(Qw),
-                           static_cast<const __nv_bfloat16 *>(K), s, workspace, st);
-        if (rc == GRAPHKV_OK)
-            rc = run_propagate(d, l, static_cast<const __nv_bfloat16 *>(K), s, nullptr, workspace, st);
-    } else {
-        rc = run_score(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), s,
-                       workspace, st);
-        if (rc == GRAPHKV_OK)
-            rc = run_propagate(d, l, static_cast<const float *>(K), s, nullptr, workspace, st);
-    }
-    if (rc != GRAPHKV_OK) return rc;
-    return run_select_gather(d, elem, s, K, V, K_out, V_out, idx_out, st);
+    if (params->dtype == GRAPHKV_BF16)
+        return do_compress(d, l, static_cast<const __nv_bfloat16 *>(Qw),
+                           static_cast<const __nv_bfloat16 *>(K), V, K_out, V_out, idx_out, s,
+                           workspace, st);
+    return do_compress(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), V, K_out,
+                       V_out, idx_out, s, workspace, st);
 }
 
 graphkv_status graphkv_read_status(const void *workspace, void *stream)

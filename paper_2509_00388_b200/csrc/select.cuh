@@ -76,10 +76,16 @@ __global__ void __launch_bounds__(kSelectThreads) topk_select_kernel(SelectArgs 
                 valid = (u & mask) == prefix;
                 bin = (u >> shift) & 255u;
             }
+            // lanes sharing the first valid lane's digit are counted with one atomic; the others
+            // add for themselves
             const unsigned vm = __ballot_sync(0xffffffffu, valid);
-            if (valid) {
-                const unsigned peers = __match_any_sync(vm, bin);
-                if (lane == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+            if (vm) {
+                const int leader = __ffs(vm) - 1;
+                const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
+                const bool same = valid && bin == lbin;
+                const unsigned sm = __ballot_sync(0xffffffffu, same);
+                if (lane == leader) atomicAdd(&hist[lbin], (uint32_t)__popc(sm));
+                else if (valid && !same) atomicAdd(&hist[bin], 1u);
             }
         }
         __syncthreads();

@@ -1,0 +1,352 @@
+// Steps (II)+(III), first half, on the tensor cores (bf16 inputs): the edges e_ij of Eq. 1 between
+// the source nodes of a head and every prefix key, and per key chunk the candidates for each
+// source's top-m neighbourhood (Eq. 3).  The edge matrix never leaves the SM.
+//
+// One CTA owns a chunk of at most 512 / NP key tiles of one head (NP = source count padded to
+// 16, 32 or 64).  Each 128-key tile arrives by TMA, one tcgen05.mma block computes its
+// 128 x NP dot products against the source keys into its own TMEM columns, and the epilogue
+// threads (thread = key) take the key's norm from the staged tile.  When the sweep is over the
+// chunk's whole edge block still sits in TMEM, and the CTA
+//   1. takes, per source, a threshold tau that at least m eligible edges of the chunk reach:
+//      the (m+1)-th largest of the per-thread maxima (distinct threads hold distinct keys, and
+//      at most one of them is the source itself);
+//   2. re-reads TMEM and lists the edges >= tau, excluding the source itself;
+//   3. if a list outgrows its capacity (many ties), finds that source's exact m-th largest
+//      (edge descending, position ascending) by bisection over counting passes and lists
+//      exactly those m.
+// The lists of all chunks hold every member of the head-wide top-m.  Each listed edge is also
+// counted in a per-source histogram over the cosine, from which the row-wise finishing kernel
+// takes a bound that leaves it a few dozen edges to rank.
+#pragma once
+
+#include "tc_common.cuh"
+
+namespace graphkv {
+namespace tc {
+
+constexpr int kSimThreads = 320;
+constexpr int kSimEpiThreads = 256;
+constexpr int kSimMaxNeighbors = 32;    // m this path handles
+constexpr int kSimMaxTiles = 32;        // tiles per CTA at NP = 16 (512 TMEM columns)
+
+struct SimTcArgs {
+    Dims d;
+    const __nv_bfloat16 *K;
+    const int *src;        // [units][K_src] source positions
+    Cand *cand;            // [units][K_src][chunks][kCandCap]; unused slots hold e = kCandEmpty
+    uint32_t *cand_hist;   // [units][K_src][kCandBins] listed edges per cosine bin (zeroed before)
+    int *status;
+    int unit0;
+    int chunks;            // CTAs per unit
+    int n_tiles;           // 128-key tiles per unit
+    int stages;
+};
+
+template <int NP> __host__ __device__ constexpr int sim_tiles_cap() { return 512 / NP; }
+
+// Dynamic shared memory (1024-byte aligned base):
+//   [0, NP*256)                      source keys, K-major 128-byte swizzle (two 64-column halves)
+//   [.., + stages*32 KB)             key tiles in flight; reused for the per-thread maxima
+//   barriers, inverse norms of the chunk's keys, source bookkeeping, candidate lists
+template <int NP> __host__ __device__ inline size_t sim_smem_bytes(int stages)
+{
+    return 1024 + (size_t)NP * 256 + (size_t)stages * kTileBytes + (8 + 8 + kSimMaxTiles) * 8 + 16 +
+           (size_t)sim_tiles_cap<NP>() * 128 * 4 + (size_t)NP * 4 * 4 + (size_t)NP * kCandCap * 8 + 64;
+}
+
+template <int NP>
+__device__ __forceinline__ void tmem_ld_np(uint32_t taddr, float (&v)[NP])
+{
+    if constexpr (NP == 16) {
+        tmem_ld16(taddr, v);
+    } else {
+#pragma unroll
+        for (int c = 0; c < NP / 32; ++c) {
+            float t[32];
+            tmem_ld32(taddr + c * 32, t);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[c * 32 + i] = t[i];
+        }
+    }
+}
+
+template <int NP>
+__global__ void __launch_bounds__(kSimThreads, 1)
+similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int kTilesCap = sim_tiles_cap<NP>();
+    const Dims &d = a.d;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t s_src = base;
+    const uint32_t s_stage0 = s_src + NP * 256;
+    const uint32_t s_full0 = s_stage0 + a.stages * kTileBytes;
+    const uint32_t s_empty0 = s_full0 + 8 * 8;
+    const uint32_t s_done0 = s_empty0 + 8 * 8;
+    const uint32_t s_tmem = s_done0 + kSimMaxTiles * 8;
+    const uint32_t s_invn = s_tmem + 16;
+    const uint32_t s_book = s_invn + kTilesCap * 128 * 4;
+    const uint32_t s_list = s_book + NP * 4 * 4;
+    float *inv_norm = reinterpret_cast<float *>(gen + (s_invn - base));        // [tile][128]
+    int *src_pos = reinterpret_cast<int *>(gen + (s_book - base));              // [NP]
+    float *src_inv = reinterpret_cast<float *>(src_pos + NP);                   // [NP]
+    uint32_t *tau = reinterpret_cast<uint32_t *>(src_inv + NP);                 // [NP]
+    int *cnt = reinterpret_cast<int *>(tau + NP);                               // [NP]
+    Cand *list = reinterpret_cast<Cand *>(gen + (s_list - base));               // [NP][kCandCap]
+    uint32_t *thread_max = reinterpret_cast<uint32_t *>(gen + (s_stage0 - base));  // [NP][256]
+    int *xchg = reinterpret_cast<int *>(gen + (s_tmem - base)) + 2;             // 2 words
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int unit = a.unit0 + blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
+    const int chunk = blockIdx.x;
+    const int per = a.n_tiles / a.chunks, rem = a.n_tiles % a.chunks;
+    const int t0 = chunk * per + min(chunk, rem);
+    const int n_local = per + (chunk < rem ? 1 : 0);
+    const __nv_bfloat16 *Kh = a.K + b * d.ks[0] + (long long)h * d.ks[1];
+    const int *src = a.src + (long long)unit * d.K_src;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < a.stages; ++i) {
+            mbar_init(s_full0 + 8 * i, 1);
+            mbar_init(s_empty0 + 8 * i, 1 + 4);       // MMA commit + the four norm warps of a tile
+        }
+        for (int i = 0; i < kSimMaxTiles; ++i) mbar_init(s_done0 + 8 * i, 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK);
+    }
+    if (warp == 1) {
+        tmem_alloc(s_tmem, 512);
+        tmem_relinquish();
+    }
+    // source keys -> swizzled operand rows (rows >= K_src are zero), their positions and norms
+    for (int i = threadIdx.x; i < NP * 16; i += blockDim.x) {
+        const int r = i >> 4, c16 = i & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (r < d.K_src) v = *reinterpret_cast<const uint4 *>(Kh + (long long)src[r] * d.ks[2] + c16 * 8);
+        *reinterpret_cast<uint4 *>(gen + sw128_offset(NP, r, c16)) = v;
+    }
+    for (int r = warp; r < NP; r += kSimThreads / 32) {
+        float n2 = 0.f;
+        int pos = -1;
+        if (r < d.K_src) {
+            pos = src[r];
+            const uint2 raw = *reinterpret_cast<const uint2 *>(Kh + (long long)pos * d.ks[2] + lane * 4);
+            const float x0 = __uint_as_float(raw.x << 16), x1 = __uint_as_float(raw.x & 0xffff0000u);
+            const float x2 = __uint_as_float(raw.y << 16), x3 = __uint_as_float(raw.y & 0xffff0000u);
+            n2 = warp_sum(x0 * x0 + x1 * x1 + x2 * x2 + x3 * x3);
+        }
+        if (lane == 0) {
+            src_pos[r] = pos;
+            src_inv[r] = 1.0f / fmaxf(sqrtf(n2), kNormEps);
+            cnt[r] = 0;
+        }
+    }
+    if (threadIdx.x == 0) xchg[0] = 1;
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(gen + (s_tmem - base));
+    bool ok = true;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int i = 0; i < n_local; ++i) {
+                const int st = i % a.stages, ph = (i / a.stages) & 1;
+                if (!mbar_wait(s_empty0 + 8 * st, ph ^ 1)) { ok = false; break; }
+                const uint32_t dst = s_stage0 + st * kTileBytes;
+                mbar_expect_tx(s_full0 + 8 * st, kTileBytes);
+                tma_load_4d(dst, &tmK, s_full0 + 8 * st, 0, (t0 + i) * kTileKeys, h, b);
+                tma_load_4d(dst + kHalfBytes, &tmK, s_full0 + 8 * st, 64, (t0 + i) * kTileKeys, h, b);
+                ++issued;
+            }
+            if (!ok)        // gave up: let the copies already in flight land before the CTA exits
+                for (int i = max(0, issued - a.stages); i < issued; ++i)
+                    mbar_wait(s_full0 + 8 * (i % a.stages), (i / a.stages) & 1);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, NP);
+            for (int i = 0; i < n_local; ++i) {
+                const int st = i % a.stages, ph = (i / a.stages) & 1;
+                if (!mbar_wait(s_full0 + 8 * st, ph)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t kt = s_stage0 + st * kTileBytes;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint32_t koff = (k >> 2) * kHalfBytes + (k & 3) * 32;
+                    const uint32_t soff = (k >> 2) * (NP * 128) + (k & 3) * 32;
+                    umma_bf16(tmem_base + i * NP, umma_desc_sw128(kt + koff),
+                              umma_desc_sw128(s_src + soff), idesc, k > 0);
+                }
+                umma_commit(s_empty0 + 8 * st);
+                umma_commit(s_done0 + 8 * i);
+            }
+        }
+    } else {
+        // ---- epilogue threads: thread = key (TMEM lane); the two warp sets alternate tiles ----
+        const int quad = warp & 3, set = (warp - 2) >> 2;
+        const int key_lane = quad * 32 + lane;
+        const int et = set * 128 + key_lane;                   // epilogue thread id, 0..255
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        float best[NP];
+#pragma unroll
+        for (int c = 0; c < NP; ++c) best[c] = -2.0f;
+        bool alive = true;
+        for (int i = set; i < n_local; i += 2) {
+            const int st = i % a.stages, ph = (i / a.stages) & 1;
+            float inv = 0.f;
+            if (alive) alive = __all_sync(0xffffffffu, mbar_wait(s_full0 + 8 * st, ph));
+            if (alive) {
+                // squared norm of this thread's key from the staged tile
+                const uint8_t *tile = gen + (s_stage0 - base) + st * kTileBytes;
+                float n0 = 0.f, n1 = 0.f;
+#pragma unroll
+                for (int c16 = 0; c16 < 16; ++c16) {
+                    const uint4 raw = *reinterpret_cast<const uint4 *>(tile + sw128_offset(128, key_lane, c16));
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float lo = __uint_as_float(w[q] << 16), hi = __uint_as_float(w[q] & 0xffff0000u);
+                        n0 = fmaf(lo, lo, n0);
+                        n1 = fmaf(hi, hi, n1);
+                    }
+                }
+                inv = 1.0f / fmaxf(sqrtf(n0 + n1), kNormEps);
+                inv_norm[i * 128 + key_lane] = inv;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_empty0 + 8 * st);
+                alive = __all_sync(0xffffffffu, mbar_wait(s_done0 + 8 * i, 0));
+            }
+            if (alive) {
+                tc_fence_after();
+                float v[NP];
+                tmem_ld_np<NP>(lane_addr + i * NP, v);
+                if ((t0 + i) * kTileKeys + key_lane < d.N) {
+#pragma unroll
+                    for (int c = 0; c < NP; ++c) {
+                        const float e = fminf(fmaxf(v[c] * inv * src_inv[c], -1.0f), 1.0f);
+                        best[c] = fmaxf(best[c], e);
+                    }
+                }
+            }
+        }
+        ok = alive;
+        // every tile's copies and MMAs are complete once both sets are here: the stage memory is free
+        if (!alive && lane == 0) xchg[0] = 0;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        const bool all_alive = xchg[0] != 0;
+        if (all_alive) {
+#pragma unroll
+            for (int c = 0; c < NP; ++c) thread_max[c * kSimEpiThreads + et] = float_to_key(best[c]);
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            // 1. thresholds: warp w of the eight takes sources w, w + 8, ...
+            const int ew = warp - 2;
+            for (int c = ew; c < d.K_src; c += 8) {
+                uint32_t v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = thread_max[c * kSimEpiThreads + q * 32 + lane];
+                uint32_t prefix = 0;
+                for (int bit = 31; bit >= 13; --bit) {
+                    const uint32_t cand = prefix | (1u << bit);
+                    int n = 0;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) n += __popc(__ballot_sync(0xffffffffu, v[q] >= cand));
+                    if (n >= d.m + 1) prefix = cand;
+                }
+                if (lane == 0) tau[c] = prefix;
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            // 2. list the edges that reach the threshold
+            uint32_t thr[NP];
+#pragma unroll
+            for (int c = 0; c < NP; ++c) thr[c] = c < d.K_src ? tau[c] : 0xffffffffu;
+            for (int i = set; i < n_local; i += 2) {
+                const int j = (t0 + i) * kTileKeys + key_lane;
+                const float inv = inv_norm[i * 128 + key_lane];
+                float v[NP];
+                tmem_ld_np<NP>(lane_addr + i * NP, v);
+                if (j < d.N) {
+#pragma unroll
+                    for (int c = 0; c < NP; ++c) {
+                        const float e = fminf(fmaxf(v[c] * inv * src_inv[c], -1.0f), 1.0f);
+                        if (float_to_key(e) >= thr[c] && j != src_pos[c]) {
+                            const int pos = atomicAdd(&cnt[c], 1);
+                            if (pos < kCandCap) list[c * kCandCap + pos] = Cand{e, j};
+                        }
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            // 3. a list that outgrew its capacity: exact m-th largest (edge desc, position asc)
+            for (int c = 0; c < d.K_src; ++c) {
+                if (cnt[c] <= kCandCap) continue;                 // uniform: shared memory value
+                unsigned long long t64 = 0ull;
+                const float sinv = src_inv[c];
+                const int self = src_pos[c];
+                for (int bit = 63; bit >= 0; --bit) {
+                    const unsigned long long cand = t64 | (1ull << bit);
+                    int n = 0;
+                    for (int i = set; i < n_local; i += 2) {
+                        const int j = (t0 + i) * kTileKeys + key_lane;
+                        const float dot = tmem_ld1(lane_addr + i * NP + c);
+                        const float e = fminf(fmaxf(dot * inv_norm[i * 128 + key_lane] * sinv, -1.0f), 1.0f);
+                        n += (j < d.N && j != self && edge_key(e, j) >= cand) ? 1 : 0;
+                    }
+                    n = __reduce_add_sync(0xffffffffu, n);
+                    if (et == 0) xchg[bit & 1] = 0;
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (lane == 0 && n) atomicAdd(&xchg[bit & 1], n);
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (xchg[bit & 1] >= d.m) t64 = cand;
+                }
+                if (et == 0) cnt[c] = 0;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                for (int i = set; i < n_local; i += 2) {
+                    const int j = (t0 + i) * kTileKeys + key_lane;
+                    const float dot = tmem_ld1(lane_addr + i * NP + c);
+                    const float e = fminf(fmaxf(dot * inv_norm[i * 128 + key_lane] * sinv, -1.0f), 1.0f);
+                    if (j < d.N && j != self && edge_key(e, j) >= t64) {
+                        const int pos = atomicAdd(&cnt[c], 1);
+                        if (pos < kCandCap) list[c * kCandCap + pos] = Cand{e, j};
+                    }
+                }
+                if (et == 0) tau[c] = static_cast<uint32_t>(t64 >> 32);
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+            }
+            // write the lists out (unused slots marked empty) and count the listed edges per bin
+            for (int c = 0; c < d.K_src; ++c) {
+                const long long slot = ((long long)unit * d.K_src + c) * a.chunks + chunk;
+                const int n = min(cnt[c], kCandCap);
+                if (et < kCandCap) {
+                    Cand cd{kCandEmpty, -1};
+                    if (et < n) {
+                        cd = list[c * kCandCap + et];
+                        atomicAdd(a.cand_hist + ((long long)unit * d.K_src + c) * kCandBins + cand_bin(cd.e), 1u);
+                    }
+                    a.cand[slot * kCandCap + et] = cd;
+                }
+            }
+        } else {
+            // a wait ran out: publish empty lists so the merge reads nothing undefined
+            for (int i = et; i < d.K_src * kCandCap; i += kSimEpiThreads) {
+                const long long slot = ((long long)unit * d.K_src + i / kCandCap) * a.chunks + chunk;
+                a.cand[slot * kCandCap + i % kCandCap] = Cand{kCandEmpty, -1};
+            }
+        }
+        tc_fence_before();
+    }
+    if (!ok && a.status) atomicExch(a.status, (int)GRAPHKV_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace tc
+}  // namespace graphkv
