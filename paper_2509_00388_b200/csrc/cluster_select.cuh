@@ -332,6 +332,7 @@ struct PoolSelectArgs {
     int *src_out;          // [units][k] ascending positions
     uint32_t *zero;        // optional: [units][zero_words] words this launch clears for later kernels
     int zero_words;
+    int wait_prior;        // launched with programmatic stream serialization
 };
 
 // grid = units * C CTAs in clusters of C; block kThreads.
@@ -347,6 +348,8 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
     const int n_local = max(0, min(a.chunk, N - base));
     float *vals = s.vals + a.halo;
     float *row_s = a.s + (long long)unit * N;
+    if (a.wait_prior) pdl_wait();
+    pdl_launch_dependents();
     if (a.zero)
         for (int i = rank * kThreads + tid; i < a.zero_words; i += C * kThreads)
             a.zero[(long long)unit * a.zero_words + i] = 0u;
@@ -406,6 +409,7 @@ struct FinishArgs {
     int elem_bytes;
     const unsigned char *K, *V;
     unsigned char *K_out, *V_out;
+    int wait_prior;            // launched with programmatic stream serialization
 };
 
 // grid = units * C CTAs in clusters of C; block kThreads.
@@ -422,6 +426,8 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     const int n_local = max(0, min(a.chunk, N - base));
     float *vals = s.vals;
     float *row_s = a.s + (long long)unit * N;
+    if (a.wait_prior) pdl_wait();
+    pdl_launch_dependents();
     for (int i = tid; i < n_local; i += kThreads) vals[i] = row_s[base + i];
     __syncthreads();
 

@@ -77,6 +77,17 @@ __device__ __forceinline__ unsigned long long edge_key(float e, int j)
            static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(j));
 }
 
+// Programmatic dependent launch: let the next kernel of the stream start its prologue, and wait
+// (in that next kernel) until the kernels before it have completed and their writes are visible.
+__device__ __forceinline__ void pdl_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll

@@ -26,6 +26,8 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Workspace carve-up; every region starts 256-byte aligned.
 struct Layout {
     size_t status;      // int status word (256 bytes reserved)
+    size_t arrivals;    // stats CTAs done per unit [units] (directly after the status word)
+    size_t row_c;       // softmax row constants [units][GW]
     size_t part;        // softmax row statistics per key chunk
     size_t a;           // attention mass before pooling [units][N]
     size_t s;           // scores when the caller gives no array [units][N]
@@ -124,8 +126,10 @@ Layout layout_of(const Dims &d)
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     l.n_stat_chunks = ceil_div(d.L, kStatsChunk);
-    l.max_parts = l.n_stat_chunks > 2 * 148 ? l.n_stat_chunks : 2 * 148;
+    l.max_parts = l.n_stat_chunks > 148 ? l.n_stat_chunks : 148;
     l.status = take(kAlign);
+    l.arrivals = take((size_t)d.units * sizeof(int));
+    l.row_c = take((size_t)d.units * d.GW * sizeof(float));
     l.part = take((size_t)d.units * l.max_parts * d.GW * 2 * sizeof(float));
     l.a = take((size_t)d.units * d.N * sizeof(float));
     l.s = take((size_t)d.units * d.N * sizeof(float));
@@ -200,6 +204,55 @@ struct LaunchScope {
 template <typename T> inline T *at(void *ws, size_t off)
 {
     return reinterpret_cast<T *>(static_cast<unsigned char *>(ws) + off);
+}
+
+// ---- launches with attributes -------------------------------------------------------------------
+// Kernels of one API call after the first are launched with programmatic stream serialization:
+// their prologue (barriers, TMEM, operand staging, the first key tiles) overlaps the tail of the
+// kernel before, and they execute griddepcontrol.wait before touching anything an earlier kernel
+// of the call wrote.
+thread_local int t_launches_in_call = 0;
+
+inline bool next_launch_is_dependent()
+{
+    static const bool enabled = [] { const char *v = getenv("GRAPHKV_PDL"); return v ? atoi(v) != 0 : true; }();
+    const bool dep = enabled && t_launches_in_call > 0 && !g_trace_on.load(std::memory_order_relaxed);
+    ++t_launches_in_call;
+    return dep;
+}
+
+template <typename... KArgs, typename... Args>
+graphkv_status launch_ex(const char *name, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                         cudaStream_t st, bool dependent, int cluster_x, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (dependent) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    cudaError_t e;
+    GKV_LAUNCH(name, st, (e = cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...)));
+    if (e != cudaSuccess) {
+        if (getenv("GRAPHKV_LOG")) fprintf(stderr, "graphkv: %s: %s\n", name, cudaGetErrorString(e));
+        return GRAPHKV_ERR_CUDA;
+    }
+    return GRAPHKV_OK;
 }
 
 // ---- step (I) ------------------------------------------------------------------------------
@@ -282,41 +335,37 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
     const int rows_pad = 128 * row_tiles;
     const int stages = row_tiles == 1 ? 5 : 4;
     const size_t smem = tc::score_smem_bytes(rows_pad, stages);
-    static bool attr = false;
-    if (!attr) {
-        const size_t mx = tc::score_smem_bytes(256, 4) > tc::score_smem_bytes(128, 5)
-                              ? tc::score_smem_bytes(256, 4) : tc::score_smem_bytes(128, 5);
-        if (!set_smem(tc::score_stats_tc<1>, mx) || !set_smem(tc::score_stats_tc<2>, mx) ||
-            !set_smem(tc::score_emit_tc<1>, mx) || !set_smem(tc::score_emit_tc<2>, mx))
-            return GRAPHKV_ERR_CUDA;
-        attr = true;
-    }
+    static std::once_flag once;
+    static bool attr_ok = true;
+    std::call_once(once, [] {
+        const size_t mx = std::max(tc::score_smem_bytes(256, 4), tc::score_smem_bytes(128, 5));
+        attr_ok = set_smem(tc::score_stats_tc<1>, mx) && set_smem(tc::score_stats_tc<2>, mx) &&
+                  set_smem(tc::score_emit_tc<1>, mx) && set_smem(tc::score_emit_tc<2>, mx);
+    });
+    if (!attr_ok) return GRAPHKV_ERR_CUDA;
     const int n_sms = 148;
     const int tiles_stats = ceil_div(d.L, tc::kTileKeys), tiles_emit = ceil_div(d.N, tc::kTileKeys);
     const int group = units_per_group(d);
-    for (int u0 = 0; u0 < d.units; u0 += group) {
+    graphkv_status rc = GRAPHKV_OK;
+    for (int u0 = 0; u0 < d.units && rc == GRAPHKV_OK; u0 += group) {
         const int nu = std::min(group, d.units - u0);
         int chunks_s = std::max(1, std::min(n_sms / nu, tiles_stats));
-        chunks_s = std::min(chunks_s, l.max_parts / 2);
+        chunks_s = std::min(chunks_s, l.max_parts);
         const int chunks_e = std::max(1, std::min(n_sms / nu, tiles_emit));
-        tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), a, at<int>(ws, l.status), u0, chunks_s,
-                           tiles_stats, 2 * chunks_s, stages};
+        tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), at<float>(ws, l.row_c), at<int>(ws, l.arrivals), a,
+                           at<int>(ws, l.status), u0, chunks_s, tiles_stats, chunks_s, stages, 0};
         tc::ScoreTcArgs ea = sa;
         ea.chunks = chunks_e;
         ea.n_tiles = tiles_emit;
-        if (row_tiles == 1) {
-            GKV_LAUNCH("score_stats_tc", st,
-                       (tc::score_stats_tc<1><<<dim3(chunks_s, nu), tc::kScoreThreads, smem, st>>>(tmK, sa)));
-            GKV_LAUNCH("score_emit_tc", st,
-                       (tc::score_emit_tc<1><<<dim3(chunks_e, nu), tc::kScoreThreads, smem, st>>>(tmK, ea)));
-        } else {
-            GKV_LAUNCH("score_stats_tc", st,
-                       (tc::score_stats_tc<2><<<dim3(chunks_s, nu), tc::kScoreThreads, smem, st>>>(tmK, sa)));
-            GKV_LAUNCH("score_emit_tc", st,
-                       (tc::score_emit_tc<2><<<dim3(chunks_e, nu), tc::kScoreThreads, smem, st>>>(tmK, ea)));
-        }
+        sa.wait_prior = next_launch_is_dependent();
+        rc = launch_ex("score_stats_tc", row_tiles == 1 ? tc::score_stats_tc<1> : tc::score_stats_tc<2>,
+                       dim3(chunks_s, nu), dim3(tc::kScoreThreads), smem, st, sa.wait_prior != 0, 1, tmK, sa);
+        if (rc != GRAPHKV_OK) break;
+        ea.wait_prior = next_launch_is_dependent();
+        rc = launch_ex("score_emit_tc", row_tiles == 1 ? tc::score_emit_tc<1> : tc::score_emit_tc<2>,
+                       dim3(chunks_e, nu), dim3(tc::kScoreThreads), smem, st, ea.wait_prior != 0, 1, tmK, ea);
     }
-    return launch_status();
+    return rc;
 }
 
 inline graphkv_status run_mass(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
@@ -347,8 +396,8 @@ ClusterPlan cluster_plan(const Dims &d)
     return p;
 }
 
-template <typename Kern, typename Args>
-graphkv_status launch_cluster(const char *name, Kern kern, const Args &args, int clusters, int C,
+template <typename Args>
+graphkv_status launch_cluster(const char *name, void (*kern)(Args), Args args, int clusters, int C,
                               size_t smem, cudaStream_t st)
 {
     static std::once_flag once;
@@ -358,25 +407,9 @@ graphkv_status launch_cluster(const char *name, Kern kern, const Args &args, int
         attr_ok = set_smem(cs::pool_select_kernel, mx) && set_smem(cs::finish_kernel, mx);
     });
     if (!attr_ok) return GRAPHKV_ERR_CUDA;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(clusters * C);
-    cfg.blockDim = dim3(cs::kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = C;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e;
-    GKV_LAUNCH(name, st, (e = cudaLaunchKernelEx(&cfg, kern, args)));
-    if (e != cudaSuccess) {
-        if (getenv("GRAPHKV_LOG")) fprintf(stderr, "graphkv: %s: %s\n", name, cudaGetErrorString(e));
-        return GRAPHKV_ERR_CUDA;
-    }
-    return GRAPHKV_OK;
+    args.wait_prior = next_launch_is_dependent();
+    return launch_ex(name, kern, dim3(clusters * C), dim3(cs::kThreads), smem, st, args.wait_prior != 0, C,
+                     args);
 }
 
 // Pooling of a -> s (when a != nullptr) and the k source nodes of Eq. 2 (when k > 0).
@@ -387,7 +420,7 @@ graphkv_status run_pool_sources(const Dims &d, const float *a, float *s, int k, 
     if (!a && k == 0) return GRAPHKV_OK;
     const ClusterPlan cp = cluster_plan(d);
     if (cp.ok) {
-        cs::PoolSelectArgs pa{d, cp.C, cp.chunk, a ? cp.halo : 0, 0, a, s, k, src, zero, zero_words};
+        cs::PoolSelectArgs pa{d, cp.C, cp.chunk, a ? cp.halo : 0, 0, a, s, k, src, zero, zero_words, 0};
         return launch_cluster(a ? (k ? "pool_select_sources" : "pool_max") : "select_sources",
                               cs::pool_select_kernel, pa, d.units, cp.C,
                               cs::smem_bytes(cp.chunk, pa.halo), st);
@@ -430,19 +463,22 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *
             const int nu = std::min(group, d.units - u0);
             tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(K), src, at<Cand>(ws, l.cand),
                              at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
-                             sp.n_tiles, sp.stages};
-            const dim3 grid(sp.chunks, nu);
+                             sp.n_tiles, sp.stages, 0};
+            sa.wait_prior = next_launch_is_dependent();
+            const dim3 grid(sp.chunks, nu), block(tc::kSimThreads);
+            graphkv_status rc;
             if (sp.NP == 16)
-                GKV_LAUNCH("similarity_tc", st,
-                           (tc::similarity_tc<16><<<grid, tc::kSimThreads, tc::sim_smem_bytes<16>(sp.stages), st>>>(tmK, sa)));
+                rc = launch_ex("similarity_tc", tc::similarity_tc<16>, grid, block,
+                               tc::sim_smem_bytes<16>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
             else if (sp.NP == 32)
-                GKV_LAUNCH("similarity_tc", st,
-                           (tc::similarity_tc<32><<<grid, tc::kSimThreads, tc::sim_smem_bytes<32>(sp.stages), st>>>(tmK, sa)));
+                rc = launch_ex("similarity_tc", tc::similarity_tc<32>, grid, block,
+                               tc::sim_smem_bytes<32>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
             else
-                GKV_LAUNCH("similarity_tc", st,
-                           (tc::similarity_tc<64><<<grid, tc::kSimThreads, tc::sim_smem_bytes<64>(sp.stages), st>>>(tmK, sa)));
+                rc = launch_ex("similarity_tc", tc::similarity_tc<64>, grid, block,
+                               tc::sim_smem_bytes<64>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
+            if (rc != GRAPHKV_OK) return rc;
         }
-        return launch_status();
+        return GRAPHKV_OK;
     }
     float *sims = at<float>(ws, l.sims);
     GKV_LAUNCH("similarity_simt", st,
@@ -467,7 +503,7 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, float 
                           has_graph ? 1 : 0, has_graph && merge ? 1 : 0, at<Cand>(ws, l.cand),
                           at<uint32_t>(ws, l.cand_hist), sim_plan(d, true).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
                           static_cast<const unsigned char *>(K), static_cast<const unsigned char *>(V),
-                          static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out)};
+                          static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0};
         const char *name = has_graph ? (do_select ? "decay_select_gather" : "decay_rounds") : "select_gather";
         return launch_cluster(name, cs::finish_kernel, fa, d.units, cp.C, cs::smem_bytes(cp.chunk, 0), st);
     }
@@ -493,10 +529,18 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, float 
 }
 
 // ---- the calls, typed ---------------------------------------------------------------------------
+// Status word and arrival counters start every scoring call at zero.
+inline graphkv_status reset_words(const Dims &d, const Layout &l, void *ws, cudaStream_t st)
+{
+    return cudaMemsetAsync(ws, 0, l.arrivals + (size_t)d.units * sizeof(int), st) == cudaSuccess
+               ? GRAPHKV_OK : GRAPHKV_ERR_CUDA;
+}
+
 template <typename T>
 graphkv_status do_score(const Dims &d, const Layout &l, const T *Q, const T *K, float *scores,
                         void *ws, cudaStream_t st)
 {
+    if (reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
     float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
     graphkv_status rc = run_mass(d, l, Q, K, a, ws, st);
     if (rc != GRAPHKV_OK || d.kp == 1) return rc;
@@ -525,6 +569,7 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
                            cudaStream_t st)
 {
     const bool graph = graph_active(d);
+    if (reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
     float *a = d.kp > 1 ? at<float>(ws, l.a) : s;
     graphkv_status rc = run_mass(d, l, Q, K, a, ws, st);
     if (rc != GRAPHKV_OK) return rc;
@@ -564,6 +609,7 @@ graphkv_status graphkv_score(const graphkv_params *params, const void *Qw, const
     Dims d;
     graphkv_status rc = resolve(params, &d);
     if (rc != GRAPHKV_OK) return rc;
+    t_launches_in_call = 0;
     if (!Qw || !K || !scores || !aligned16(Qw) || !aligned16(K)) return GRAPHKV_ERR_INVALID_ARG;
     const Layout l = layout_of(d);
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
@@ -582,6 +628,7 @@ graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, fl
     Dims d;
     graphkv_status rc = resolve(params, &d);
     if (rc != GRAPHKV_OK) return rc;
+    t_launches_in_call = 0;
     if (!K || !scores || !aligned16(K)) return GRAPHKV_ERR_INVALID_ARG;
     const Layout l = layout_of(d);
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
@@ -600,6 +647,7 @@ graphkv_status graphkv_select_gather(const graphkv_params *params, const float *
     Dims d;
     graphkv_status rc = resolve(params, &d);
     if (rc != GRAPHKV_OK) return rc;
+    t_launches_in_call = 0;
     if (!scores || !idx_out) return GRAPHKV_ERR_INVALID_ARG;
     if ((K == nullptr) != (K_out == nullptr) || (V == nullptr) != (V_out == nullptr))
         return GRAPHKV_ERR_INVALID_ARG;
@@ -620,6 +668,7 @@ graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, co
     Dims d;
     graphkv_status rc = resolve(params, &d);
     if (rc != GRAPHKV_OK) return rc;
+    t_launches_in_call = 0;
     if (!Qw || !K || !V || !K_out || !V_out || !idx_out) return GRAPHKV_ERR_INVALID_ARG;
     if (!aligned16(Qw) || !aligned16(K) || !aligned16(V) || !aligned16(K_out) || !aligned16(V_out))
         return GRAPHKV_ERR_INVALID_ARG;

@@ -24,14 +24,17 @@ constexpr int kEpiWarps = 8;
 struct ScoreTcArgs {
     Dims d;
     const __nv_bfloat16 *Q;
-    float *part;        // [units][n_parts][GW][2] row statistics (max, sum) per key chunk
+    float *part;        // [units][stats_chunks][GW][2] row statistics (max, sum) per key chunk
+    float *row_c;       // [units][GW] c_r = max_r + log2(Z_r), written by the last stats CTA of a unit
+    int *arrivals;      // [units] stats CTAs done per unit (zero before the launch; reset on the way)
     float *a_out;       // [units][N] attention mass before pooling
     int *status;        // workspace status word
     int unit0;          // first unit of this launch
     int chunks;         // key chunks (CTAs) per unit
     int n_tiles;        // 128-key tiles per unit in this sweep
-    int n_parts;        // partial statistics per row (stats sweep: 2 * its chunks)
+    int stats_chunks;   // key chunks of the statistics sweep (partials per row)
     int stages;         // shared-memory K tiles in flight
+    int wait_prior;     // launched with programmatic stream serialization: wait for the kernels before
 };
 
 struct ScoreSmem {
@@ -59,24 +62,83 @@ __device__ __forceinline__ ScoreSmem score_smem_layout(uint8_t *raw, int rows_pa
 __host__ __device__ inline size_t score_smem_bytes(int rows_pad, int stages)
 {
     return 1024 + (size_t)rows_pad * 256 + (size_t)stages * kTileBytes + 8 * 8 * 2 + 2 * 8 * 2 + 16 +
-           (size_t)(rows_pad + 2 * 128) * 4 + 64;
+           8192 + 64;      // 8 KB: the CTA's row statistics / row constants and the exchange buffer
 }
 
-// Q rows of the unit -> K-major swizzled operand (rows >= GW zero-filled).
+// Q rows of the unit -> K-major swizzled operand (rows >= GW zero-filled).  Threads tid of
+// nthreads; loads are issued four at a time ahead of the shared-memory stores.
 __device__ __forceinline__ void stage_q(uint8_t *q_gen, int rows_pad, const Dims &d,
-                                        const __nv_bfloat16 *Q, int b, int h)
+                                        const __nv_bfloat16 *Q, int b, int h, int tid, int nthreads)
 {
-    for (int i = threadIdx.x; i < rows_pad * 16; i += blockDim.x) {
-        const int r = i >> 4, c16 = i & 15;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < d.GW) {
-            const int g = r / d.W, rw = r % d.W;
-            const __nv_bfloat16 *qp =
-                Q + b * d.qs[0] + (long long)(h * d.G + g) * d.qs[1] + rw * d.qs[2] + c16 * 8;
-            v = *reinterpret_cast<const uint4 *>(qp);
+    const __nv_bfloat16 *Qh = Q + b * d.qs[0] + (long long)(h * d.G) * d.qs[1];
+    for (int i0 = tid; i0 < rows_pad * 16; i0 += 4 * nthreads) {
+        uint4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = i0 + k * nthreads;
+            const int r = i >> 4, c16 = i & 15;
+            v[k] = make_uint4(0, 0, 0, 0);
+            if (i < rows_pad * 16 && r < d.GW) {
+                const int g = r / d.W, rw = r - g * d.W;
+                v[k] = *reinterpret_cast<const uint4 *>(Qh + g * d.qs[1] + rw * d.qs[2] + c16 * 8);
+            }
         }
-        *reinterpret_cast<uint4 *>(q_gen + sw128_offset(rows_pad, r, c16)) = v;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = i0 + k * nthreads;
+            if (i < rows_pad * 16)
+                *reinterpret_cast<uint4 *>(q_gen + sw128_offset(rows_pad, i >> 4, i & 15)) = v[k];
+        }
     }
+}
+
+// Barriers and TMEM of both sweeps, then the CTA synchronised so that every warp may use them.
+// Returns the TMEM base address.
+__device__ __forceinline__ uint32_t score_setup(const ScoreSmem &s, uint8_t *gen, const CUtensorMap *tmK,
+                                                int stages, uint32_t tmem_cols)
+{
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < stages; ++i) {
+            mbar_init(s.full0 + 8 * i, 1);
+            mbar_init(s.empty0 + 8 * i, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(s.tfull0 + 8 * i, 1);
+            mbar_init(s.tempty0 + 8 * i, 8);       // the eight epilogue warps
+        }
+        mbar_fence_init();
+        tma_prefetch_desc(tmK);
+    }
+    if ((threadIdx.x >> 5) == 1) {
+        tmem_alloc(s.tmem_slot, tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    return *reinterpret_cast<volatile uint32_t *>(gen + (s.tmem_slot - s.q));
+}
+
+// TMA producer (one thread): key tiles t0+i of (h, b), i in [i_begin, i_end), into the stage ring.
+// The keys are an input of the call, so the producer never waits for the kernels before.
+__device__ __forceinline__ bool score_produce(const ScoreSmem &s, const CUtensorMap *tmK, int stages,
+                                              int t0, int i_begin, int i_end, int h, int b)
+{
+    bool ok = true;
+    int issued = i_begin;
+    for (int i = i_begin; i < i_end; ++i) {
+        const int st = i % stages, ph = (i / stages) & 1;
+        if (!mbar_wait(s.empty0 + 8 * st, ph ^ 1)) { ok = false; break; }
+        const uint32_t dst = s.stage0 + st * kTileBytes;
+        mbar_expect_tx(s.full0 + 8 * st, kTileBytes);
+        tma_load_4d(dst, tmK, s.full0 + 8 * st, 0, (t0 + i) * kTileKeys, h, b);
+        tma_load_4d(dst + kHalfBytes, tmK, s.full0 + 8 * st, 64, (t0 + i) * kTileKeys, h, b);
+        ++issued;
+    }
+    if (!ok)        // gave up: let the copies already in flight land before the CTA exits
+        for (int i = max(0, issued - stages); i < issued; ++i)
+            mbar_wait(s.full0 + 8 * (i % stages), (i / stages) & 1);
+    return ok;
 }
 
 __device__ __forceinline__ void tile_range(int n_tiles, int chunks, int chunk, int *t0, int *t1)
@@ -125,47 +187,24 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     tile_range(a.n_tiles, a.chunks, chunk, &t0, &t1);
     const int n_local = t1 - t0;
 
-    if (threadIdx.x == 0) {
-        if (a.status && blockIdx.x == 0 && blockIdx.y == 0 && a.unit0 == 0) *a.status = 0;
-        for (int i = 0; i < a.stages; ++i) {
-            mbar_init(s.full0 + 8 * i, 1);
-            mbar_init(s.empty0 + 8 * i, 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(s.tfull0 + 8 * i, 1);
-            mbar_init(s.tempty0 + 8 * i, kEpiWarps);
-        }
-        mbar_fence_init();
-        tma_prefetch_desc(&tmK);
-    }
-    if (warp == 1) {
-        tmem_alloc(s.tmem_slot, kTmemCols);
-        tmem_relinquish();
-    }
-    stage_q(gen, kRowsPad, d, a.Q, b, h);
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(gen + (s.tmem_slot - s.q));
+    float2 *cta_part = reinterpret_cast<float2 *>(gen + (s.misc - s.q));      // [2][kRowsPad]
+    int *s_flag = reinterpret_cast<int *>(gen + (s.tmem_slot - s.q)) + 2;
+    const int n_ahead = min(n_local, a.stages);
+
+    const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols);
     bool ok = true;
+    if (warp == 0) {
+        if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b);
+    } else {
+        stage_q(gen, kRowsPad, d, a.Q, b, h, threadIdx.x - 32, kScoreThreads - 32);
+        fence_proxy_async();
+    }
+    if (a.wait_prior) pdl_wait();
+    pdl_launch_dependents();
+    __syncthreads();
 
     if (warp == 0) {
-        if (lane == 0) {
-            int issued = 0;
-            for (int i = 0; i < n_local; ++i) {
-                const int st = i % a.stages, ph = (i / a.stages) & 1;
-                if (!mbar_wait(s.empty0 + 8 * st, ph ^ 1)) { ok = false; break; }
-                const uint32_t dst = s.stage0 + st * kTileBytes;
-                mbar_expect_tx(s.full0 + 8 * st, kTileBytes);
-                tma_load_4d(dst, &tmK, s.full0 + 8 * st, 0, (t0 + i) * kTileKeys, h, b);
-                tma_load_4d(dst + kHalfBytes, &tmK, s.full0 + 8 * st, 64, (t0 + i) * kTileKeys, h, b);
-                ++issued;
-            }
-            if (!ok)        // gave up: let the copies already in flight land before the CTA exits
-                for (int i = max(0, issued - a.stages); i < issued; ++i)
-                    mbar_wait(s.full0 + 8 * (i % a.stages), (i / a.stages) & 1);
-        }
+        if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b);
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
@@ -233,14 +272,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         }
         ok = alive;
 #pragma unroll
-        for (int rt = 0; rt < kRowTiles; ++rt) {
-            const int r = rt * 128 + row;
-            if (r < d.GW) {
-                float *o = a.part + (((long long)unit * a.n_parts + chunk * 2 + set) * d.GW + r) * 2;
-                o[0] = mx[rt];
-                o[1] = z[rt];
-            }
-        }
+        for (int rt = 0; rt < kRowTiles; ++rt) cta_part[set * kRowsPad + rt * 128 + row] = make_float2(mx[rt], z[rt]);
     }
     if (!ok && a.status) atomicExch(a.status, (int)GRAPHKV_ERR_TIMEOUT);
     tc_fence_before();
@@ -249,6 +281,40 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
+    }
+    // this CTA's statistics of each row; the last CTA of the unit to get here merges all chunks
+    // into the unit's row constants c_r
+    for (int r = threadIdx.x; r < d.GW; r += kScoreThreads) {
+        const float2 p0 = cta_part[r], p1 = cta_part[kRowsPad + r];
+        const float mx = fmaxf(p0.x, p1.x);
+        reinterpret_cast<float2 *>(a.part)[((long long)unit * a.stats_chunks + chunk) * d.GW + r] =
+            make_float2(mx, p0.y * ex2(p0.x - mx) + p1.y * ex2(p1.x - mx));
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *s_flag = atomicAdd(a.arrivals + unit, 1) == a.chunks - 1;
+    __syncthreads();
+    if (*s_flag) {
+        __threadfence();
+        const float2 *pu = reinterpret_cast<const float2 *>(a.part) + (long long)unit * a.stats_chunks * d.GW;
+        for (int r = threadIdx.x; r < d.GW; r += kScoreThreads) {
+            float mx = kNegBig, z = 0.f;
+            for (int q0 = 0; q0 < a.chunks; q0 += 8) {       // eight loads in flight at a time
+                float2 v[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    v[k] = q0 + k < a.chunks ? __ldcg(pu + (long long)(q0 + k) * d.GW + r)
+                                             : make_float2(kNegBig, 0.f);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float mn = fmaxf(mx, v[k].x);
+                    z = z * ex2(mx - mn) + v[k].y * ex2(v[k].x - mn);
+                    mx = mn;
+                }
+            }
+            a.row_c[(long long)unit * d.GW + r] = mx + log2f(z);
+        }
+        if (threadIdx.x == 0) a.arrivals[unit] = 0;      // ready for the next launch
     }
 }
 
@@ -274,60 +340,24 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     const int n_local = t1 - t0;
     const int n_cols = (d.GW + 31) & ~31;            // UMMA N: every x32 slice read below is written
 
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < a.stages; ++i) {
-            mbar_init(s.full0 + 8 * i, 1);
-            mbar_init(s.empty0 + 8 * i, 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(s.tfull0 + 8 * i, 1);
-            mbar_init(s.tempty0 + 8 * i, kEpiWarps);
-        }
-        mbar_fence_init();
-        tma_prefetch_desc(&tmK);
-    }
-    if (warp == 1) {
-        tmem_alloc(s.tmem_slot, kTmemCols);
-        tmem_relinquish();
-    }
-    stage_q(gen, kRowsPad, d, a.Q, b, h);
-    // merge the per-chunk statistics of each row: c_r = max_r + log2(sum_r)
-    for (int r = threadIdx.x; r < kRowsPad; r += blockDim.x) {
-        float c = INFINITY;                          // padding rows contribute 2^-inf = 0
-        if (r < d.GW) {
-            const float *p = a.part + ((long long)unit * a.n_parts * d.GW + r) * 2;
-            float mx = kNegBig;
-            for (int q = 0; q < a.n_parts; ++q) mx = fmaxf(mx, p[(long long)q * d.GW * 2]);
-            float z = 0.f;
-            for (int q = 0; q < a.n_parts; ++q)
-                z += p[(long long)q * d.GW * 2 + 1] * ex2(p[(long long)q * d.GW * 2] - mx);
-            c = mx + log2f(z);
-        }
-        row_c[r] = c;
-    }
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(gen + (s.tmem_slot - s.q));
+    const int n_ahead = min(n_local, a.stages);
+    const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols);
     bool ok = true;
+    if (warp == 0) {
+        if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b);
+    } else {
+        stage_q(gen, kRowsPad, d, a.Q, b, h, threadIdx.x - 32, kScoreThreads - 32);
+        fence_proxy_async();
+    }
+    if (a.wait_prior) pdl_wait();
+    pdl_launch_dependents();
+    // c_r of the unit's rows; padding rows contribute 2^-inf = 0
+    for (int r = threadIdx.x; r < kRowsPad; r += kScoreThreads)
+        row_c[r] = r < d.GW ? __ldcg(a.row_c + (long long)unit * d.GW + r) : INFINITY;
+    __syncthreads();
 
     if (warp == 0) {
-        if (lane == 0) {
-            int issued = 0;
-            for (int i = 0; i < n_local; ++i) {
-                const int st = i % a.stages, ph = (i / a.stages) & 1;
-                if (!mbar_wait(s.empty0 + 8 * st, ph ^ 1)) { ok = false; break; }
-                const uint32_t dst = s.stage0 + st * kTileBytes;
-                mbar_expect_tx(s.full0 + 8 * st, kTileBytes);
-                tma_load_4d(dst, &tmK, s.full0 + 8 * st, 0, (t0 + i) * kTileKeys, h, b);
-                tma_load_4d(dst + kHalfBytes, &tmK, s.full0 + 8 * st, 64, (t0 + i) * kTileKeys, h, b);
-                ++issued;
-            }
-            if (!ok)        // gave up: let the copies already in flight land before the CTA exits
-                for (int i = max(0, issued - a.stages); i < issued; ++i)
-                    mbar_wait(s.full0 + 8 * (i % a.stages), (i / a.stages) & 1);
-        }
+        if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b);
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(128, n_cols);

@@ -40,6 +40,7 @@ struct SimTcArgs {
     int chunks;            // CTAs per unit
     int n_tiles;           // 128-key tiles per unit
     int stages;
+    int wait_prior;        // launched with programmatic stream serialization
 };
 
 template <int NP> __host__ __device__ constexpr int sim_tiles_cap() { return 512 / NP; }
@@ -119,6 +120,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         tmem_alloc(s_tmem, 512);
         tmem_relinquish();
     }
+    if (a.wait_prior) pdl_wait();
+    pdl_launch_dependents();
     // source keys -> swizzled operand rows (rows >= K_src are zero), their positions and norms
     for (int i = threadIdx.x; i < NP * 16; i += blockDim.x) {
         const int r = i >> 4, c16 = i & 15;
