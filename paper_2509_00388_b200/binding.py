@@ -14,7 +14,7 @@ from typing import Optional, Tuple
 import torch
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libgraphkv.so")
+LIB_PATH = os.environ.get("GRAPHKV_LIB") or os.path.join(HERE, "libgraphkv.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 BF16, F32 = 0, 1

@@ -322,6 +322,26 @@ __device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chu
     __syncwarp();
 }
 
+// vals[i] = row[base + i] for i in [lo, hi) (positions outside [0, N) read as `fill`), all threads
+// of the CTA, eight loads in flight per thread ahead of the shared-memory stores.
+__device__ __forceinline__ void load_chunk(const float *row, int base, int lo, int hi, int N,
+                                           float *vals, float fill)
+{
+    for (int i0 = lo + (int)threadIdx.x; i0 < hi; i0 += 8 * kThreads) {
+        float r[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int i = i0 + k * kThreads, j = base + i;
+            r[k] = (i < hi && j >= 0 && j < N) ? __ldcg(row + j) : fill;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int i = i0 + k * kThreads;
+            if (i < hi) vals[i] = r[k];
+        }
+    }
+}
+
 struct PoolSelectArgs {
     Dims d;
     int C, chunk, halo;
@@ -356,10 +376,7 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
     if (a.a) {
         const float *row_a = a.a + (long long)unit * N;
         const int half = a.halo;
-        for (int i = tid - half; i < n_local + half; i += kThreads) {
-            const int j = base + i;
-            vals[i] = (n_local > 0 && j >= 0 && j < N) ? row_a[j] : -INFINITY;
-        }
+        if (n_local > 0) load_chunk(row_a, base, -half, n_local + half, N, vals, -INFINITY);
         __syncthreads();
         float pooled[kMaxPerThread];
 #pragma unroll
@@ -381,7 +398,7 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
             }
         }
     } else {
-        for (int i = tid; i < n_local; i += kThreads) vals[i] = row_s[base + i];
+        load_chunk(row_s, base, 0, n_local, N, vals, 0.f);
     }
     __syncthreads();
     if (a.k > 0) {
@@ -428,7 +445,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     float *row_s = a.s + (long long)unit * N;
     if (a.wait_prior) pdl_wait();
     pdl_launch_dependents();
-    for (int i = tid; i < n_local; i += kThreads) vals[i] = row_s[base + i];
+    load_chunk(row_s, base, 0, n_local, N, vals, 0.f);
     __syncthreads();
 
     if (a.has_graph && a.merge) {
@@ -504,20 +521,33 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
             const long long row_bytes = (long long)kHeadDim * a.elem_bytes;
             const int b = unit / d.hkv, h = unit % d.hkv;
             const long long total = (long long)rows_out * vec_per_row;
-            for (long long p = (long long)rank * kThreads + tid; p < total; p += (long long)C * kThreads) {
-                const int c = (int)(p % vec_per_row);
-                const int t = (int)(p / vec_per_row);
-                const int src_row = t < d.B ? __ldcg(idx + t) : N + (t - d.B);
-                const long long dst = ((long long)unit * rows_out + t) * row_bytes + c * 16;
-                if (a.K) {
-                    const long long off = (b * d.ks[0] + h * d.ks[1] + src_row * d.ks[2]) * a.elem_bytes;
-                    *reinterpret_cast<uint4 *>(a.K_out + dst) =
-                        *reinterpret_cast<const uint4 *>(a.K + off + c * 16);
+            const long long stride = (long long)C * kThreads;
+            for (long long p0 = (long long)rank * kThreads + tid; p0 < total; p0 += 4 * stride) {
+                uint4 kv[4], vv[4];
+                long long dst[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const long long p = p0 + u * stride;
+                    dst[u] = -1;
+                    if (p < total) {
+                        const int c = (int)(p % vec_per_row);
+                        const int t = (int)(p / vec_per_row);
+                        const int src_row = t < d.B ? __ldcg(idx + t) : N + (t - d.B);
+                        dst[u] = ((long long)unit * rows_out + t) * row_bytes + c * 16;
+                        if (a.K)
+                            kv[u] = *reinterpret_cast<const uint4 *>(
+                                a.K + (b * d.ks[0] + h * d.ks[1] + src_row * d.ks[2]) * a.elem_bytes + c * 16);
+                        if (a.V)
+                            vv[u] = *reinterpret_cast<const uint4 *>(
+                                a.V + (b * d.vs[0] + h * d.vs[1] + src_row * d.vs[2]) * a.elem_bytes + c * 16);
+                    }
                 }
-                if (a.V) {
-                    const long long off = (b * d.vs[0] + h * d.vs[1] + src_row * d.vs[2]) * a.elem_bytes;
-                    *reinterpret_cast<uint4 *>(a.V_out + dst) =
-                        *reinterpret_cast<const uint4 *>(a.V + off + c * 16);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (dst[u] >= 0) {
+                        if (a.K) *reinterpret_cast<uint4 *>(a.K_out + dst[u]) = kv[u];
+                        if (a.V) *reinterpret_cast<uint4 *>(a.V_out + dst[u]) = vv[u];
+                    }
                 }
             }
         }

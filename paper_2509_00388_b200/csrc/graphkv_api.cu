@@ -87,14 +87,36 @@ int env_int(const char *name, int dflt)
     return v ? atoi(v) : dflt;
 }
 
-// Units per launch group: the group's keys should stay in L2 between the sweeps.
+// Units per launch of a sweep.  By default all units go into one launch: measured on B200, the
+// fixed cost of extra launches outweighs serving the later sweeps of a small group from L2
+// (GRAPHKV_L2_GROUP_MB bounds the keys of a group for experiments).
 int units_per_group(const Dims &d)
 {
     const double mb = (double)d.L * kHeadDim * 2 / 1.0e6;
-    int n = (int)(env_int("GRAPHKV_L2_GROUP_MB", 72) / mb);
+    int n = (int)(env_int("GRAPHKV_L2_GROUP_MB", 1 << 20) / mb);
     if (n < 1) n = 1;
     if (n > d.units) n = d.units;
     return n;
+}
+
+// Key chunks (CTAs) per unit for a sweep of `tiles` key tiles per unit over `units` units, one CTA
+// per SM: the count that minimises waves x (tiles per CTA + a per-CTA overhead of about three
+// tile times), with at least min_chunks and at most max_chunks.
+int sweep_chunks(int units, int tiles, int min_chunks, int max_chunks)
+{
+    const int n_sms = 148;
+    int best = std::max(1, min_chunks);
+    long long best_cost = -1;
+    const int hi = std::max(best, std::min(tiles, max_chunks));
+    for (int c = best; c <= hi; ++c) {
+        const long long waves = ceil_div(units * c, n_sms);
+        const long long cost = waves * (ceil_div(tiles, c) + 3);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = c;
+        }
+    }
+    return best;
 }
 
 // Tensor-core similarity sweep: usable for bf16 keys, up to 64 sources and 32 neighbours.
@@ -115,7 +137,7 @@ SimPlan sim_plan(const Dims &d, bool bf16)
     p.stages = p.NP == 64 ? 4 : 5;
     const int cap = 512 / p.NP;
     const int group = units_per_group(d);
-    p.chunks = std::max(ceil_div(p.n_tiles, cap), std::max(1, std::min(148 / group, p.n_tiles)));
+    p.chunks = sweep_chunks(group, p.n_tiles, ceil_div(p.n_tiles, cap), 1 << 20);
     p.ok = true;
     return p;
 }
@@ -343,15 +365,13 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
                   set_smem(tc::score_emit_tc<1>, mx) && set_smem(tc::score_emit_tc<2>, mx);
     });
     if (!attr_ok) return GRAPHKV_ERR_CUDA;
-    const int n_sms = 148;
     const int tiles_stats = ceil_div(d.L, tc::kTileKeys), tiles_emit = ceil_div(d.N, tc::kTileKeys);
     const int group = units_per_group(d);
     graphkv_status rc = GRAPHKV_OK;
     for (int u0 = 0; u0 < d.units && rc == GRAPHKV_OK; u0 += group) {
         const int nu = std::min(group, d.units - u0);
-        int chunks_s = std::max(1, std::min(n_sms / nu, tiles_stats));
-        chunks_s = std::min(chunks_s, l.max_parts);
-        const int chunks_e = std::max(1, std::min(n_sms / nu, tiles_emit));
+        const int chunks_s = sweep_chunks(nu, tiles_stats, 1, l.max_parts);
+        const int chunks_e = sweep_chunks(nu, tiles_emit, 1, 1 << 20);
         tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), at<float>(ws, l.row_c), at<int>(ws, l.arrivals), a,
                            at<int>(ws, l.status), u0, chunks_s, tiles_stats, chunks_s, stages, 0};
         tc::ScoreTcArgs ea = sa;

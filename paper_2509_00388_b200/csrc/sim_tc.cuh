@@ -8,8 +8,9 @@
 // threads (thread = key) take the key's norm from the staged tile.  When the sweep is over the
 // chunk's whole edge block still sits in TMEM, and the CTA
 //   1. takes, per source, a threshold tau that at least m eligible edges of the chunk reach:
-//      the (m+1)-th largest of the per-thread maxima (distinct threads hold distinct keys, and
-//      at most one of them is the source itself);
+//      the lower edge of the highest cosine bin such that m+1 of the per-thread maxima lie in or
+//      above it (distinct threads hold distinct keys, and at most one of them is the source
+//      itself);
 //   2. re-reads TMEM and lists the edges >= tau, excluding the source itself;
 //   3. if a list outgrows its capacity (many ties), finds that source's exact m-th largest
 //      (edge descending, position ascending) by bisection over counting passes and lists
@@ -28,6 +29,7 @@ constexpr int kSimThreads = 320;
 constexpr int kSimEpiThreads = 256;
 constexpr int kSimMaxNeighbors = 32;    // m this path handles
 constexpr int kSimMaxTiles = 32;        // tiles per CTA at NP = 16 (512 TMEM columns)
+constexpr int kMaxBins = 256;           // cosine bins over [-1, 1] for the per-thread maxima
 
 struct SimTcArgs {
     Dims d;
@@ -92,10 +94,11 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     float *inv_norm = reinterpret_cast<float *>(gen + (s_invn - base));        // [tile][128]
     int *src_pos = reinterpret_cast<int *>(gen + (s_book - base));              // [NP]
     float *src_inv = reinterpret_cast<float *>(src_pos + NP);                   // [NP]
-    uint32_t *tau = reinterpret_cast<uint32_t *>(src_inv + NP);                 // [NP]
+    float *tau = src_inv + NP;                                                  // [NP] threshold cosine
     int *cnt = reinterpret_cast<int *>(tau + NP);                               // [NP]
     Cand *list = reinterpret_cast<Cand *>(gen + (s_list - base));               // [NP][kCandCap]
-    uint32_t *thread_max = reinterpret_cast<uint32_t *>(gen + (s_stage0 - base));  // [NP][256]
+    uint32_t *max_hist = reinterpret_cast<uint32_t *>(gen + (s_stage0 - base)); // [NP][kMaxBins], after the sweep
+    Cand *own = reinterpret_cast<Cand *>(gen + (s_stage0 - base));              // [NP][256][slots], after max_hist
     int *xchg = reinterpret_cast<int *>(gen + (s_tmem - base)) + 2;             // 2 words
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -194,9 +197,9 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         const int key_lane = quad * 32 + lane;
         const int et = set * 128 + key_lane;                   // epilogue thread id, 0..255
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        float best[NP];
+        float best[NP];                     // per source: max over this thread's keys of dot / |k_j|
 #pragma unroll
-        for (int c = 0; c < NP; ++c) best[c] = -2.0f;
+        for (int c = 0; c < NP; ++c) best[c] = -INFINITY;
         bool alive = true;
         for (int i = set; i < n_local; i += 2) {
             const int st = i % a.stages, ph = (i / a.stages) & 1;
@@ -229,10 +232,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 tmem_ld_np<NP>(lane_addr + i * NP, v);
                 if ((t0 + i) * kTileKeys + key_lane < d.N) {
 #pragma unroll
-                    for (int c = 0; c < NP; ++c) {
-                        const float e = fminf(fmaxf(v[c] * inv * src_inv[c], -1.0f), 1.0f);
-                        best[c] = fmaxf(best[c], e);
-                    }
+                    for (int c = 0; c < NP; ++c) best[c] = fmaxf(best[c], v[c] * inv);
                 }
             }
         }
@@ -242,45 +242,139 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         asm volatile("bar.sync 1, 256;" ::: "memory");
         const bool all_alive = xchg[0] != 0;
         if (all_alive) {
-#pragma unroll
-            for (int c = 0; c < NP; ++c) thread_max[c * kSimEpiThreads + et] = float_to_key(best[c]);
+            // 1. thresholds.  The cosine of a thread's best key for source c is the rounded product
+            //    of its best dot / |k_j| with 1 / |k_c| (rounding is monotone); histogram those over
+            //    [-1, 1] and take the lower edge of the highest bin with m+1 maxima in or above it.
+            for (int i = et; i < d.K_src * kMaxBins; i += kSimEpiThreads) max_hist[i] = 0u;
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            // 1. thresholds: warp w of the eight takes sources w, w + 8, ...
-            const int ew = warp - 2;
-            for (int c = ew; c < d.K_src; c += 8) {
-                uint32_t v[8];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) v[q] = thread_max[c * kSimEpiThreads + q * 32 + lane];
-                uint32_t prefix = 0;
-                for (int bit = 31; bit >= 13; --bit) {
-                    const uint32_t cand = prefix | (1u << bit);
-                    int n = 0;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) n += __popc(__ballot_sync(0xffffffffu, v[q] >= cand));
-                    if (n >= d.m + 1) prefix = cand;
+            for (int c = 0; c < NP; ++c) {
+                if (c < d.K_src && best[c] > -INFINITY) {
+                    const float e = fminf(fmaxf(best[c] * src_inv[c], -1.0f), 1.0f);
+                    const int bin = min(max(static_cast<int>((e + 1.0f) * (kMaxBins / 2)), 0), kMaxBins - 1);
+                    atomicAdd(&max_hist[c * kMaxBins + bin], 1u);
                 }
-                if (lane == 0) tau[c] = prefix;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            // 2. list the edges that reach the threshold
-            uint32_t thr[NP];
+            const int ew = warp - 2;
+            for (int c = ew; c < d.K_src; c += 8) {
+                constexpr int kPer = kMaxBins / 32;          // lane l holds bins [l * kPer, (l + 1) * kPer)
+                uint32_t hb[kPer], mine = 0;
 #pragma unroll
-            for (int c = 0; c < NP; ++c) thr[c] = c < d.K_src ? tau[c] : 0xffffffffu;
+                for (int q = 0; q < kPer; ++q) {
+                    hb[q] = max_hist[c * kMaxBins + lane * kPer + q];
+                    mine += hb[q];
+                }
+                uint32_t above = 0;                          // maxima in the lanes above this one
+                for (int l = 31; l > 0; --l) {
+                    const uint32_t t = __shfl_sync(0xffffffffu, mine, l);
+                    if (lane < l) above += t;
+                }
+                int bstar = -1;
+                uint32_t run = above;
+#pragma unroll
+                for (int q = kPer - 1; q >= 0; --q) {
+                    run += hb[q];
+                    if (bstar < 0 && run >= (uint32_t)(d.m + 1)) bstar = lane * kPer + q;
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) bstar = max(bstar, __shfl_xor_sync(0xffffffffu, bstar, o));
+                if (lane == 0) tau[c] = bstar <= 0 ? -1.0f : (float)bstar * (2.0f / kMaxBins) - 1.0f;
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            // 2. list the edges that reach the threshold.  theta is the threshold brought to the scale
+            //    of dot / |k_j|, lowered by a few ulps so that no edge with cosine >= tau is missed.
+            //    Branch-free: a thread's first kSlots edges of a source go to slots of its own by
+            //    predicated stores (2-bit counters packed in registers); only threads with more
+            //    edges of one source than that come back for them below.
+            constexpr int kSlots = NP <= 32 ? 2 : 1;
+            float theta[NP];
+#pragma unroll
+            for (int c = 0; c < NP; ++c) {
+                const float q = c < d.K_src ? tau[c] / src_inv[c] : INFINITY;
+                theta[c] = q - fabsf(q) * 2.4e-7f - 1e-30f;
+            }
+            uint32_t nfound[NP / 16];                  // 2 bits per source: edges found, saturating at 3
+#pragma unroll
+            for (int w = 0; w < NP / 16; ++w) nfound[w] = 0u;
             for (int i = set; i < n_local; i += 2) {
                 const int j = (t0 + i) * kTileKeys + key_lane;
-                const float inv = inv_norm[i * 128 + key_lane];
+                const float inv = j < d.N ? inv_norm[i * 128 + key_lane] : 0.f;
                 float v[NP];
                 tmem_ld_np<NP>(lane_addr + i * NP, v);
-                if (j < d.N) {
 #pragma unroll
-                    for (int c = 0; c < NP; ++c) {
-                        const float e = fminf(fmaxf(v[c] * inv * src_inv[c], -1.0f), 1.0f);
-                        if (float_to_key(e) >= thr[c] && j != src_pos[c]) {
+                for (int c = 0; c < NP; ++c) {
+                    const float t = v[c] * inv;
+                    const uint32_t n = (nfound[c / 16] >> (2 * (c % 16))) & 3u;
+                    const bool pass = j < d.N && t >= theta[c];
+                    if (pass && n < kSlots) own[(c * kSimEpiThreads + et) * kSlots + n] = Cand{t, j};
+                    if (pass && n < 3u) nfound[c / 16] += 1u << (2 * (c % 16));
+                }
+            }
+            uint32_t over = 0;                         // sources of which this thread has more edges
+#pragma unroll
+            for (int c = 0; c < NP; ++c) {
+                const uint32_t n = (nfound[c / 16] >> (2 * (c % 16))) & 3u;
+#pragma unroll
+                for (int q = 0; q < kSlots; ++q)
+                    if (c < d.K_src && n <= (uint32_t)q) own[(c * kSimEpiThreads + et) * kSlots + q] = Cand{0.f, -1};
+                if (c < 32 && n > (uint32_t)kSlots) over |= 1u << (c & 31);
+                if (NP > 32 && c >= 32 && n > (uint32_t)kSlots) over |= 1u << (c & 31);   // approximate: see below
+            }
+            // the rare threads with more edges of a source than slots: rescan that source's column and
+            // append all but the first kSlots through the shared counter
+            uint32_t any_over = over;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) any_over |= __shfl_xor_sync(0xffffffffu, any_over, o);
+            for (int c = 0; c < d.K_src && any_over; ++c) {
+                if (!((any_over >> (c & 31)) & 1u)) continue;
+                const float sinv = src_inv[c];
+                const float q = tau[c] / sinv;
+                const float th = q - fabsf(q) * 2.4e-7f - 1e-30f;
+                const bool mine = (over >> (c & 31)) & 1u;
+                int skip = kSlots;
+                for (int i = set; i < n_local; i += 2) {
+                    const int j = (t0 + i) * kTileKeys + key_lane;
+                    const float t = tmem_ld1(lane_addr + i * NP + c) * (j < d.N ? inv_norm[i * 128 + key_lane] : 0.f);
+                    if (mine && j < d.N && t >= th) {
+                        if (skip > 0) --skip;
+                        else {
                             const int pos = atomicAdd(&cnt[c], 1);
-                            if (pos < kCandCap) list[c * kCandCap + pos] = Cand{e, j};
+                            if (pos < kCandCap) list[c * kCandCap + pos] = Cand{t, j};
                         }
                     }
                 }
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            // gather the threads' own slots into the lists, now as cosines: warp w takes sources
+            // w, w + 8, ...; entries the counter path added before are converted in place first
+            for (int c = ew; c < d.K_src; c += 8) {
+                const int self = src_pos[c];
+                const float sinv = src_inv[c], tc = tau[c];
+                const int n_pre = min(cnt[c], kCandCap);
+                __syncwarp();
+                for (int i = lane; i < n_pre; i += 32) {
+                    Cand cd = list[c * kCandCap + i];
+                    cd.e = fminf(fmaxf(cd.e * sinv, -1.0f), 1.0f);
+                    if (cd.e < tc || cd.j == self) cd.e = kCandEmpty;     // dropped later as empty
+                    list[c * kCandCap + i] = cd;
+                }
+                __syncwarp();
+                int basep = cnt[c];
+                __syncwarp();
+                constexpr int kPerLane = kSimEpiThreads * kSlots / 32;
+                int total = 0;
+#pragma unroll 4
+                for (int q = 0; q < kPerLane; ++q) {
+                    Cand cd = own[c * kSimEpiThreads * kSlots + q * 32 + lane];
+                    const float e = fminf(fmaxf(cd.e * sinv, -1.0f), 1.0f);
+                    const bool valid = cd.j >= 0 && cd.j != self && e >= tc;
+                    const unsigned bm = __ballot_sync(0xffffffffu, valid);
+                    const int pos = basep + total + __popc(bm & ((1u << lane) - 1u));
+                    if (valid && pos < kCandCap) list[c * kCandCap + pos] = Cand{e, cd.j};
+                    total += __popc(bm);
+                }
+                if (lane == 0) cnt[c] = basep + total;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             // 3. a list that outgrew its capacity: exact m-th largest (edge desc, position asc)
@@ -316,7 +410,6 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                         if (pos < kCandCap) list[c * kCandCap + pos] = Cand{e, j};
                     }
                 }
-                if (et == 0) tau[c] = static_cast<uint32_t>(t64 >> 32);
                 asm volatile("bar.sync 1, 256;" ::: "memory");
             }
             // write the lists out (unused slots marked empty) and count the listed edges per bin

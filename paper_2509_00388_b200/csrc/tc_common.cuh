@@ -183,6 +183,20 @@ __device__ __forceinline__ float tmem_ld1(uint32_t taddr)
     return __uint_as_float(r);
 }
 
+// Split form of the one-column load: issue several, then tmem_ld_fence over their registers.
+__device__ __forceinline__ void tmem_ld1_issue(uint32_t taddr, uint32_t &r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+}
+// Waits for every TMEM load of this thread; the empty statements tie the registers to the wait so
+// that no use of them can be scheduled above it.
+template <int N> __device__ __forceinline__ void tmem_ld_fence(uint32_t (&r)[N])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int k = 0; k < N; ++k) asm volatile("" : "+r"(r[k]));
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
