@@ -140,6 +140,34 @@ def test_exact_duplicate_keys_tie_break_like_the_oracle(gk):
     check(gk, cfg, strict_overlap=False)
 
 
+def test_identical_keys_take_the_exact_tie_paths(gk):
+    # every key of a head is the same vector: all cosines tie, so each source's neighbourhood is
+    # decided by position alone (the m lowest positions other than the source itself) and the
+    # candidate lists of every key chunk overflow into their exact bisection paths
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=5000, budget=200, n_q_heads=4, n_kv_heads=2,
+                    n_clusters=8, topk_nodes=16, neighbors=32, rounds=1, pool_kernel=1)
+    inp = wl.make_inputs(cfg)
+    K = inp["K"].clone()
+    K[:, :, :, :] = K[:, :, :1, :]
+    kw = cfg_kwargs(cfg)
+    staged = run_staged(gk, inp["Qw"], K, inp["V"], **kw)
+    fused = run_fused(gk, inp["Qw"], K, inp["V"], **kw)
+    for name in ("idx", "K_out", "V_out", "scores"):
+        assert torch.equal(staged[name].view(torch.uint8), fused[name].view(torch.uint8))
+    n = cfg.n_prefix
+    for h in range(cfg.n_kv_heads):
+        s0 = staged["scores0"][0, h]
+        o_s, o_src, o_nbr, _ = okv.propagate_unit(K[0, h], s0, n, cfg.topk_nodes, cfg.neighbors,
+                                                  cfg.rounds, cfg.decay)
+        assert sorted(staged["src"][0, h].tolist()) == sorted(o_src.tolist())
+        changed = set(torch.nonzero(staged["scores"][0, h] != s0).flatten().tolist())
+        want = set(o_nbr.flatten().tolist())
+        assert changed == {j for j in want if float(s0[j]) != 0.0}
+        assert pu.score_rel_err(staged["scores"][0, h][None], o_s[None]) <= pu.SCORE_RTOL
+        want_idx = np.sort(okv.topk(staged["scores"][0, h], cfg.budget).numpy())
+        assert np.array_equal(staged["idx"][0, h].numpy(), want_idx)
+
+
 def test_strided_inputs(gk):
     # K and V as views of a [batch, L, heads, D] buffer (token-major, the layout of a fused
     # QKV projection): strides are not those of a dense [b, h, L, D] tensor
