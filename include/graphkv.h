@@ -43,7 +43,9 @@ typedef enum {
     GRAPHKV_ERR_UNSUPPORTED = 2,   /* valid but not implemented (head_dim != 128, G*W > 256, ...) */
     GRAPHKV_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small                 */
     GRAPHKV_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                          */
-    GRAPHKV_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out (read_status only)      */
+    GRAPHKV_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out (read_status only)      */
+    GRAPHKV_ERR_BUILTIN_SCRATCH = 6 /* graphkv_score_noalloc: the problem needs more scratch than
+                                      the library's built-in array holds                         */
 } graphkv_status;
 
 typedef enum { GRAPHKV_BF16 = 0, GRAPHKV_F32 = 1 } graphkv_dtype;
@@ -87,6 +89,38 @@ int32_t graphkv_resolve_neighbors(int32_t n_prefix, int32_t neighbors);
 graphkv_status graphkv_score(const graphkv_params *params, const void *Qw, const void *K,
                              float *scores, void *workspace, size_t workspace_bytes,
                              void *stream);
+
+/* graphkv_score for callers that cannot provide a workspace.  (The paper has no counterpart: this
+ * entry point exists for the way some programs embed the library.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated -- inside a region that
+ * a framework has closed to cudaMalloc (its caching allocator is being recorded or is locked),
+ * in a hook or callback invoked from such a region, or in a process whose memory budget was
+ * handed out in full at start-up.  Such callers still own Qw, K and the `scores` output, but
+ * have nowhere to get the scratch that graphkv_score takes as `workspace`.
+ *
+ * What it does: the same kernels as graphkv_score, with the scratch (status word, per-chunk
+ * softmax statistics, row constants, the attention mass before pooling) placed in an array that
+ * is part of the library image: GRAPHKV_BUILTIN_SCRATCH_BYTES bytes of device memory that every
+ * GPU loading the library holds until the process exits.  It calls no cudaMalloc, cudaFree or
+ * allocating library routine.  Results are bit-identical to graphkv_score.
+ *
+ * Limits and rules:
+ *   - graphkv_builtin_scratch_needed(params) must not exceed GRAPHKV_BUILTIN_SCRATCH_BYTES;
+ *     otherwise nothing is launched and GRAPHKV_ERR_BUILTIN_SCRATCH is returned (for bf16
+ *     inputs with pooling the need is about 4 * batch * n_kv_heads * N bytes plus 1.5 MB).
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps what the last call left: the call
+ *     clears the words that must start at zero itself, but two calls whose kernels overlap on
+ *     the GPU (different streams, no ordering between them) race on it.  Order them.
+ *   - The device-side status word lives in the array too: graphkv_read_status_noalloc(stream)
+ *     reads it.  */
+#define GRAPHKV_BUILTIN_SCRATCH_BYTES (16u << 20)
+size_t graphkv_builtin_scratch_needed(const graphkv_params *params);
+graphkv_status graphkv_score_noalloc(const graphkv_params *params, const void *Qw, const void *K,
+                                     float *scores, void *stream);
+graphkv_status graphkv_read_status_noalloc(void *stream);
 
 /* Steps (II)+(III), "Build Graph" and "Decay Signal Propagation" (Eq. 1-5, Algorithms 1-2):
  * sources = top-k of `scores`; e_ij = cosine(k_i, k_j) for each source i and every prefix j != i;

@@ -16,13 +16,15 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("GRAPHKV_LIB") or os.path.join(HERE, "libgraphkv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BUILTIN_SCRATCH = range(7)
+BUILTIN_SCRATCH_BYTES = 16 << 20
 BF16, F32 = 0, 1
 
 EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_score",
            "graphkv_propagate", "graphkv_select_gather", "graphkv_compress",
            "graphkv_read_status", "graphkv_status_string", "graphkv_launch_count",
-           "graphkv_trace_enable", "graphkv_trace_read")
+           "graphkv_trace_enable", "graphkv_trace_read", "graphkv_builtin_scratch_needed",
+           "graphkv_score_noalloc", "graphkv_read_status_noalloc")
 
 
 class GraphKVError(RuntimeError):
@@ -73,6 +75,12 @@ def lib() -> C.CDLL:
         L.graphkv_compress.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.graphkv_read_status.restype = C.c_int
         L.graphkv_read_status.argtypes = [vp, vp]
+        L.graphkv_builtin_scratch_needed.restype = sz
+        L.graphkv_builtin_scratch_needed.argtypes = [P]
+        L.graphkv_score_noalloc.restype = C.c_int
+        L.graphkv_score_noalloc.argtypes = [P, vp, vp, vp, vp]
+        L.graphkv_read_status_noalloc.restype = C.c_int
+        L.graphkv_read_status_noalloc.argtypes = [vp]
         L.graphkv_status_string.restype = C.c_char_p
         L.graphkv_status_string.argtypes = [C.c_int]
         L.graphkv_launch_count.restype = C.c_int64
@@ -154,6 +162,22 @@ def graphkv_score(p: Params, Qw: torch.Tensor, K: torch.Tensor, scores: torch.Te
                   ws: torch.Tensor) -> None:
     _check(lib().graphkv_score(C.byref(p), _ptr(Qw), _ptr(K), _ptr(scores), _ptr(ws),
                                ws.numel(), _stream(K.device)), "graphkv_score")
+
+
+def builtin_scratch_needed(p: Params) -> int:
+    return int(lib().graphkv_builtin_scratch_needed(C.byref(p)))
+
+
+def graphkv_score_noalloc(p: Params, Qw: torch.Tensor, K: torch.Tensor, scores: torch.Tensor) -> None:
+    """graphkv_score without a workspace: the scratch is the library's built-in device array, so
+    the call allocates nothing (for callers inside regions where device allocation is closed).
+    Raises GraphKVError(ERR_BUILTIN_SCRATCH) when the problem does not fit that array."""
+    _check(lib().graphkv_score_noalloc(C.byref(p), _ptr(Qw), _ptr(K), _ptr(scores),
+                                       _stream(K.device)), "graphkv_score_noalloc")
+
+
+def graphkv_read_status_noalloc(device) -> int:
+    return int(lib().graphkv_read_status_noalloc(_stream(device)))
 
 
 def graphkv_propagate(p: Params, K: torch.Tensor, scores: torch.Tensor,

@@ -603,6 +603,29 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
                       K_out, V_out, idx_out, ws, st);
 }
 
+// ---- built-in scratch for graphkv_score_noalloc ---------------------------------------------------
+// Device memory that is part of the library image.  In host code the array's name is only a handle
+// for cudaGetSymbolAddress; kernels get the address looked up once per device.
+static __device__ __align__(256) unsigned char g_builtin_scratch[GRAPHKV_BUILTIN_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_builtin_mu;
+void *g_builtin_ptr[kMaxDevices] = {};
+
+// Address of the built-in scratch on the current device (nullptr on failure).
+void *builtin_scratch()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lk(g_builtin_mu);
+    if (!g_builtin_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess) return nullptr;
+        g_builtin_ptr[dev] = p;
+    }
+    return g_builtin_ptr[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -639,6 +662,39 @@ graphkv_status graphkv_score(const graphkv_params *params, const void *Qw, const
                         static_cast<const __nv_bfloat16 *>(K), scores, workspace, st);
     return do_score(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), scores,
                     workspace, st);
+}
+
+size_t graphkv_builtin_scratch_needed(const graphkv_params *params)
+{
+    Dims d;
+    if (resolve(params, &d) != GRAPHKV_OK) return 0;
+    return layout_of(d).s;       // the scoring call uses the regions laid out before `s`
+}
+
+graphkv_status graphkv_score_noalloc(const graphkv_params *params, const void *Qw, const void *K,
+                                     float *scores, void *stream)
+{
+    Dims d;
+    graphkv_status rc = resolve(params, &d);
+    if (rc != GRAPHKV_OK) return rc;
+    t_launches_in_call = 0;
+    if (!Qw || !K || !scores || !aligned16(Qw) || !aligned16(K)) return GRAPHKV_ERR_INVALID_ARG;
+    const Layout l = layout_of(d);
+    if (l.s > GRAPHKV_BUILTIN_SCRATCH_BYTES) return GRAPHKV_ERR_BUILTIN_SCRATCH;
+    void *ws = builtin_scratch();
+    if (!ws) return GRAPHKV_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (params->dtype == GRAPHKV_BF16)
+        return do_score(d, l, static_cast<const __nv_bfloat16 *>(Qw),
+                        static_cast<const __nv_bfloat16 *>(K), scores, ws, st);
+    return do_score(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), scores, ws, st);
+}
+
+graphkv_status graphkv_read_status_noalloc(void *stream)
+{
+    void *ws = builtin_scratch();
+    if (!ws) return GRAPHKV_ERR_CUDA;
+    return graphkv_read_status(ws, stream);
 }
 
 graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, float *scores,
@@ -752,6 +808,8 @@ const char *graphkv_status_string(graphkv_status status)
         case GRAPHKV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case GRAPHKV_ERR_CUDA: return "CUDA error";
         case GRAPHKV_ERR_TIMEOUT: return "device-side wait timed out";
+        case GRAPHKV_ERR_BUILTIN_SCRATCH:
+            return "problem needs more scratch than the built-in array of graphkv_score_noalloc holds";
     }
     return "unknown status";
 }
