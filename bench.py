@@ -71,6 +71,9 @@ def algorithmic_bytes(cfg, kernel: str) -> float:
         "score_emit": units * N * D * e + q_bytes + row,
         "score_fused": k_sweep + q_bytes + row,
         "pool_max": 2 * row,
+        "pool_select_sources": 2 * row + 4 * units * Ks,
+        "decay_select_gather": 2 * row + 4 * units * B + 4 * units * (B + W) * D * e,
+        "select_gather": row + 4 * units * B + 4 * units * (B + W) * D * e,
         "select_sources": row + 4 * units * Ks,
         "similarity": units * N * D * e + units * Ks * D * e,
         "select_neighbors": 0.0,
