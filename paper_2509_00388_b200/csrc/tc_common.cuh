@@ -204,6 +204,20 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
+// 2^x for x <= 0 on the FMA and integer pipes (the MUFU unit is the ceiling of the score sweeps):
+// x = n + f with n the nearest integer and f in [-1/2, 1/2], 2^f by a cubic fitted for relative
+// error (max 1.03e-4), 2^n by adding n to the exponent field.  x is clamped at -125 (result ~0).
+__device__ __forceinline__ float ex2_poly3(float x)
+{
+    x = fmaxf(x, -125.0f);
+    const float t = x + 12582912.0f;            // 1.5 * 2^23: the integer part lands in the low mantissa bits
+    const float f = x - (t - 12582912.0f);
+    float p = fmaf(0.0549740307f, f, 0.242215246f);
+    p = fmaf(p, f, 0.693289936f);
+    p = fmaf(p, f, 1.0f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
 // Byte offset of the 16-byte piece `c16` (0..15) of row `r` inside a K-major, 128-byte-swizzled
 // operand of `rows` rows x 128 bf16: two halves of 64 columns, rows 128 bytes apart.
 __device__ __forceinline__ uint32_t sw128_offset(int rows, int r, int c16)
