@@ -355,7 +355,9 @@ struct PoolSelectArgs {
     int wait_prior;        // launched with programmatic stream serialization
 };
 
-// grid = units * C CTAs in clusters of C; block kThreads.
+// grid = units * C CTAs in clusters of C; block kThreads.  kPer >= chunk / kThreads: elements of
+// the chunk a thread pools (a power of two up to kMaxPerThread).
+template <int kPer>
 __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs a)
 {
     extern __shared__ __align__(16) uint8_t cs_smem[];
@@ -378,9 +380,9 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
         const int half = a.halo;
         if (n_local > 0) load_chunk(row_a, base, -half, n_local + half, N, vals, -INFINITY);
         __syncthreads();
-        float pooled[kMaxPerThread];
+        float pooled[kPer];
 #pragma unroll
-        for (int q = 0; q < kMaxPerThread; ++q) {
+        for (int q = 0; q < kPer; ++q) {
             const int i = q * kThreads + tid;
             if (i < n_local) {
                 float best = vals[i - half];
@@ -390,7 +392,7 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
         }
         __syncthreads();
 #pragma unroll
-        for (int q = 0; q < kMaxPerThread; ++q) {
+        for (int q = 0; q < kPer; ++q) {
             const int i = q * kThreads + tid;
             if (i < n_local) {
                 vals[i] = pooled[q];

@@ -424,7 +424,10 @@ graphkv_status launch_cluster(const char *name, void (*kern)(Args), Args args, i
     static bool attr_ok = true;
     std::call_once(once, [] {
         const size_t mx = cs::smem_bytes(cs::kMaxChunk, cs::kMaxHalo);
-        attr_ok = set_smem(cs::pool_select_kernel, mx) && set_smem(cs::finish_kernel, mx);
+        attr_ok = set_smem(cs::pool_select_kernel<1>, mx) && set_smem(cs::pool_select_kernel<2>, mx) &&
+                  set_smem(cs::pool_select_kernel<4>, mx) && set_smem(cs::pool_select_kernel<8>, mx) &&
+                  set_smem(cs::pool_select_kernel<16>, mx) && set_smem(cs::pool_select_kernel<32>, mx) &&
+                  set_smem(cs::finish_kernel, mx);
     });
     if (!attr_ok) return GRAPHKV_ERR_CUDA;
     args.wait_prior = next_launch_is_dependent();
@@ -441,9 +444,14 @@ graphkv_status run_pool_sources(const Dims &d, const float *a, float *s, int k, 
     const ClusterPlan cp = cluster_plan(d);
     if (cp.ok) {
         cs::PoolSelectArgs pa{d, cp.C, cp.chunk, a ? cp.halo : 0, 0, a, s, k, src, zero, zero_words, 0};
-        return launch_cluster(a ? (k ? "pool_select_sources" : "pool_max") : "select_sources",
-                              cs::pool_select_kernel, pa, d.units, cp.C,
-                              cs::smem_bytes(cp.chunk, pa.halo), st);
+        const char *name = a ? (k ? "pool_select_sources" : "pool_max") : "select_sources";
+        const size_t smem = cs::smem_bytes(cp.chunk, pa.halo);
+        const int per = ceil_div(cp.chunk, cs::kThreads);
+        void (*kern)(cs::PoolSelectArgs) =
+            per <= 1 ? cs::pool_select_kernel<1> : per <= 2 ? cs::pool_select_kernel<2>
+            : per <= 4 ? cs::pool_select_kernel<4> : per <= 8 ? cs::pool_select_kernel<8>
+            : per <= 16 ? cs::pool_select_kernel<16> : cs::pool_select_kernel<32>;
+        return launch_cluster(name, kern, pa, d.units, cp.C, smem, st);
     }
     if (zero && cudaMemsetAsync(zero, 0, (size_t)d.units * zero_words * 4, st) != cudaSuccess)
         return GRAPHKV_ERR_CUDA;
