@@ -30,7 +30,7 @@ constexpr int kMaxCluster = 8;
 constexpr int kMaxHalo = 64;           // (pool_kernel - 1) / 2 the pooling path handles
 constexpr int kMaxPerThread = kMaxChunk / kThreads;
 constexpr int kStage = 2048;           // neighbour-list entries staged in shared memory at a time
-constexpr int kMergeWarps = 8;         // warps of a CTA that merge candidate lists at a time
+constexpr int kMergeWarps = 8;         // groups of four warps of a CTA, one source each at a time
 constexpr int kSurvCap = 256;          // merged candidates one warp ranks in shared memory
 static_assert(kMergeWarps * kSurvCap * sizeof(Cand) <= 2 * kStage * 4, "survivors reuse the staging area");
 
@@ -222,61 +222,14 @@ __device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, cons
     }
 }
 
-// Eq. 3 for one source: the m largest edges (cosine descending, position ascending) among the
-// candidate lists its key chunks wrote.  One warp; `surv` holds kSurvCap entries of shared memory.
-// The lists together hold every member of the top-m, and `hist` counts the listed edges per cosine
-// bin: the highest bin b with at least m listed edges in bins >= b bounds the m-th largest from
-// below, so only edges with e >= b / kCandBins need ranking.
-__device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chunks, int m,
-                                 Cand *surv, int *nbr_idx, float *nbr_e)
+// The m largest edges (cosine descending, position ascending) of the lists when too many tie at
+// the bound: exact m-th largest by bisection over the lists themselves.  One warp; returns the
+// number of survivors written (m, or fewer when fewer edges are listed).
+__device__ int merge_exact(const Cand *cand, int slots, int m, Cand *surv)
 {
     const int lane = threadIdx.x & 31;
-    constexpr int kPer = kCandBins / 32;
-    // lane l holds bins [l * kPer, (l + 1) * kPer); walk down from the top bin
-    uint32_t h[kPer], mine = 0;
-#pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-        h[q] = __ldcg(hist + lane * kPer + q);
-        mine += h[q];
-    }
-    uint32_t above = 0;                       // listed edges in the lanes above this one
-    for (int l = 31; l > 0; --l) {
-        const uint32_t t = __shfl_sync(0xffffffffu, mine, l);
-        if (lane < l) above += t;
-    }
-    int bstar = -1;
-    uint32_t run = above;
-#pragma unroll
-    for (int q = kPer - 1; q >= 0; --q) {
-        run += h[q];
-        if (bstar < 0 && run >= (uint32_t)m) bstar = lane * kPer + q;
-    }
-    // the answer is the highest bin found by any lane
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) bstar = max(bstar, __shfl_xor_sync(0xffffffffu, bstar, o));
-    const float bound = bstar <= 0 ? -1.0f : (float)bstar / (float)kCandBins;
-
-    const int slots = chunks * kCandCap;
     int ns = 0;
-    for (int i0 = 0; i0 < slots; i0 += 128) {
-        unsigned long long raw[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int i = i0 + q * 32 + lane;
-            raw[q] = i < slots ? __ldcg(reinterpret_cast<const unsigned long long *>(cand + i)) : 0ull;
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int i = i0 + q * 32 + lane;
-            const Cand cd{__uint_as_float(static_cast<uint32_t>(raw[q])), static_cast<int>(raw[q] >> 32)};
-            const bool keep = i < slots && cd.e >= bound;
-            const unsigned bm = __ballot_sync(0xffffffffu, keep);
-            const int pos = ns + __popc(bm & ((1u << lane) - 1u));
-            if (keep && pos < kSurvCap) surv[pos] = cd;
-            ns += __popc(bm);
-        }
-    }
-    if (ns > kSurvCap) {
+    {
         // too many ties at the bound: exact m-th largest by bisection over the lists themselves
         unsigned long long t64 = 0ull;
         for (int bit = 63; bit >= 0; --bit) {
@@ -308,8 +261,79 @@ __device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chu
         }
     }
     __syncwarp();
+    return min(ns, kSurvCap);
+}
+
+// Eq. 3 for one source: the m largest edges (cosine descending, position ascending) among the
+// candidate lists its key chunks wrote.  One warp; `surv` holds kSurvCap entries of shared memory.
+// The lists together hold every member of the top-m, and `hist` counts the listed edges per cosine
+// bin: the highest bin b with at least m listed edges in bins >= b bounds the m-th largest from
+// below, so only edges with e >= b / kCandBins need ranking.
+__device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chunks, int m,
+                                 Cand *surv, int *ns_sh, int bar_id, int wg, int *nbr_idx, float *nbr_e)
+{
+    const int lane = threadIdx.x & 31;
+    constexpr int kPer = kCandBins / 32;
+    // lane l holds bins [l * kPer, (l + 1) * kPer); walk down from the top bin
+    uint32_t h[kPer], mine = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        h[q] = __ldcg(hist + lane * kPer + q);
+        mine += h[q];
+    }
+    uint32_t above = 0;                       // listed edges in the lanes above this one
+    for (int l = 31; l > 0; --l) {
+        const uint32_t t = __shfl_sync(0xffffffffu, mine, l);
+        if (lane < l) above += t;
+    }
+    int bstar = -1;
+    uint32_t run = above;
+#pragma unroll
+    for (int q = kPer - 1; q >= 0; --q) {
+        run += h[q];
+        if (bstar < 0 && run >= (uint32_t)m) bstar = lane * kPer + q;
+    }
+    // the answer is the highest bin found by any lane
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bstar = max(bstar, __shfl_xor_sync(0xffffffffu, bstar, o));
+    const float bound = bstar <= 0 ? -1.0f : (float)bstar / (float)kCandBins;
+
+    // the four warps of the group take interleaved blocks of 256 slots, eight loads in flight per lane
+    if (wg == 0 && lane == 0) *ns_sh = 0;
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    const int slots = chunks * kCandCap;
+    for (int i0 = wg * 256; i0 < slots; i0 += 4 * 256) {
+        unsigned long long raw[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = i0 + q * 32 + lane;
+            raw[q] = i < slots ? __ldcg(reinterpret_cast<const unsigned long long *>(cand + i)) : 0ull;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = i0 + q * 32 + lane;
+            const Cand cd{__uint_as_float(static_cast<uint32_t>(raw[q])), static_cast<int>(raw[q] >> 32)};
+            const bool keep = i < slots && cd.e >= bound;
+            const unsigned bm = __ballot_sync(0xffffffffu, keep);
+            if (bm) {
+                int basep = 0;
+                if (lane == 0) basep = atomicAdd(ns_sh, __popc(bm));
+                basep = __shfl_sync(0xffffffffu, basep, 0);
+                const int pos = basep + __popc(bm & ((1u << lane) - 1u));
+                if (keep && pos < kSurvCap) surv[pos] = cd;
+            }
+        }
+    }
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    int ns = *ns_sh;
+    if (ns > kSurvCap) {
+        if (wg == 0) ns = merge_exact(cand, slots, m, surv);
+        if (wg == 0 && lane == 0) *ns_sh = ns;
+        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+        ns = *ns_sh;
+    }
     // rank by counting: all keys are distinct (distinct positions)
-    for (int i = lane; i < ns; i += 32) {
+    for (int i = wg * 32 + lane; i < ns; i += 128) {
         const Cand me = surv[i];
         const unsigned long long k = edge_key(me.e, me.j);
         int rank = 0;
@@ -319,7 +343,7 @@ __device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chu
             nbr_e[rank] = me.e;
         }
     }
-    __syncwarp();
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // the list may be reused
 }
 
 // vals[i] = row[base + i] for i in [lo, hi) (positions outside [0, N) read as `fill`), all threads
@@ -451,18 +475,17 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     __syncthreads();
 
     if (a.has_graph && a.merge) {
-        // Eq. 3: warp w of rank r merges sources (w + kMergeWarps * t) * C + r
-        const int warp = tid >> 5;
-        if (warp < kMergeWarps) {
-            Cand *surv = reinterpret_cast<Cand *>(s.st_idx) + warp * kSurvCap;
-            for (int src = warp * C + rank; src < d.K_src; src += kMergeWarps * C) {
-                const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
-                merge_neighbours(a.cand + slot * kCandCap,
-                                 a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
-                                 a.cand_chunks, d.m, surv,
-                                 a.nbr_idx + ((long long)unit * d.K_src + src) * d.m,
-                                 a.nbr_e + ((long long)unit * d.K_src + src) * d.m);
-            }
+        // Eq. 3: the four warps of group g of rank r merge sources (g + kMergeWarps * t) * C + r
+        const int warp = tid >> 5, grp = warp >> 2, wg = warp & 3;
+        Cand *surv = reinterpret_cast<Cand *>(s.st_idx) + grp * kSurvCap;
+        int *ns_sh = reinterpret_cast<int *>(s.misc) + 8 + grp;
+        for (int src = grp * C + rank; src < d.K_src; src += kMergeWarps * C) {
+            const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
+            merge_neighbours(a.cand + slot * kCandCap,
+                             a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
+                             a.cand_chunks, d.m, surv, ns_sh, 1 + grp, wg,
+                             a.nbr_idx + ((long long)unit * d.K_src + src) * d.m,
+                             a.nbr_e + ((long long)unit * d.K_src + src) * d.m);
         }
         __threadfence();
         if (C > 1) cl.sync(); else __syncthreads();
