@@ -87,6 +87,14 @@ def algorithmic_bytes(cfg, kernel: str) -> float:
     return 0.0
 
 
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
+# summarised in profiles/kernels_llama31_8b_32k_ncu_full.md; cold cache.  Only for the workload
+# and kernels that capture covers; anything else reports null.
+NCU_TRAFFIC = {"llama31_8b_32k": {"score_stats_tc": 67.88e6, "score_emit_tc": 67.99e6,
+                                  "pool_select_sources": 1.10e6, "similarity_tc": 67.53e6,
+                                  "decay_select_gather": 4.66e6}}
+
+
 def path_bytes(cfg) -> float:
     """Algorithmic bytes of the whole path per layer: two sweeps of K (sources depend on all
     scores), the window queries, three passes over the fp32 score rows, the K/V gather."""
@@ -300,7 +308,8 @@ def run_ours(args, cfg):
     top_bytes = algorithmic_bytes(cfg, top)
     achieved = top_bytes / (kernels[top]["avg_ms"] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC.get(cfg.name, {}).get(top),
                 "peak_source": f"{peak_kind} copy bandwidth",
                 "algorithmic_bytes_per_launch": top_bytes,
                 "avg_launch_ms": kernels[top]["avg_ms"],
