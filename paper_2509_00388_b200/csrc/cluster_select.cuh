@@ -282,9 +282,14 @@ __device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chu
         mine += h[q];
     }
     uint32_t above = 0;                       // listed edges in the lanes above this one
-    for (int l = 31; l > 0; --l) {
-        const uint32_t t = __shfl_sync(0xffffffffu, mine, l);
-        if (lane < l) above += t;
+    {
+        uint32_t incl = mine;              // suffix sum over lanes, log steps
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_down_sync(0xffffffffu, incl, o);
+            if (lane + o < 32) incl += t;
+        }
+        above = incl - mine;
     }
     int bstar = -1;
     uint32_t run = above;

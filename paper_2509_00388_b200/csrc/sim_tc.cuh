@@ -126,23 +126,28 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     if (a.wait_prior) pdl_wait();
     pdl_launch_dependents();
     // source keys -> swizzled operand rows (rows >= K_src are zero), their positions and norms
-    for (int i = threadIdx.x; i < NP * 16; i += blockDim.x) {
+    // (16 consecutive threads share a row: the row's squared norm is reduced among them)
+    for (int i0 = 0; i0 < NP * 16; i0 += kSimThreads) {
+        const int i = i0 + threadIdx.x;
         const int r = i >> 4, c16 = i & 15;
+        const bool in = i < NP * 16;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < d.K_src) v = *reinterpret_cast<const uint4 *>(Kh + (long long)src[r] * d.ks[2] + c16 * 8);
-        *reinterpret_cast<uint4 *>(gen + sw128_offset(NP, r, c16)) = v;
-    }
-    for (int r = warp; r < NP; r += kSimThreads / 32) {
-        float n2 = 0.f;
         int pos = -1;
-        if (r < d.K_src) {
+        if (in && r < d.K_src) {
             pos = src[r];
-            const uint2 raw = *reinterpret_cast<const uint2 *>(Kh + (long long)pos * d.ks[2] + lane * 4);
-            const float x0 = __uint_as_float(raw.x << 16), x1 = __uint_as_float(raw.x & 0xffff0000u);
-            const float x2 = __uint_as_float(raw.y << 16), x3 = __uint_as_float(raw.y & 0xffff0000u);
-            n2 = warp_sum(x0 * x0 + x1 * x1 + x2 * x2 + x3 * x3);
+            v = *reinterpret_cast<const uint4 *>(Kh + (long long)pos * d.ks[2] + c16 * 8);
         }
-        if (lane == 0) {
+        if (in) *reinterpret_cast<uint4 *>(gen + sw128_offset(NP, r, c16)) = v;
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float n2 = 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float lo = __uint_as_float(w[q] << 16), hi = __uint_as_float(w[q] & 0xffff0000u);
+            n2 = fmaf(lo, lo, fmaf(hi, hi, n2));
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+        if (in && c16 == 0) {
             src_pos[r] = pos;
             src_inv[r] = 1.0f / fmaxf(sqrtf(n2), kNormEps);
             cnt[r] = 0;
@@ -266,9 +271,14 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                     mine += hb[q];
                 }
                 uint32_t above = 0;                          // maxima in the lanes above this one
-                for (int l = 31; l > 0; --l) {
-                    const uint32_t t = __shfl_sync(0xffffffffu, mine, l);
-                    if (lane < l) above += t;
+                {
+                    uint32_t incl = mine;              // suffix sum over lanes, log steps
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t t = __shfl_down_sync(0xffffffffu, incl, o);
+                        if (lane + o < 32) incl += t;
+                    }
+                    above = incl - mine;
                 }
                 int bstar = -1;
                 uint32_t run = above;
