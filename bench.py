@@ -318,7 +318,11 @@ def run_ours(args, cfg):
                                "achieved_gbs": path_bytes(cfg) / (ms_step * 1e-3) / 1e9,
                                "frac_of_peak": path_bytes(cfg) / (ms_step * 1e-3) / 1e9 / peak,
                                "frac_of_8tbs": path_bytes(cfg) / (ms_step * 1e-3) / 1e9 / 8000.0},
-                "kernels": {n: round(k["ms_per_step"], 5) for n, k in kernels.items()}}
+                "kernels": {n: round(k["ms_per_step"], 5) for n, k in kernels.items()},
+                "per_kernel": {n: {"algorithmic_bytes": algorithmic_bytes(cfg, n),
+                                   "achieved_gbs": round(algorithmic_bytes(cfg, n) / (k["avg_ms"] * 1e-3) / 1e9, 1),
+                                   "frac": round(algorithmic_bytes(cfg, n) / (k["avg_ms"] * 1e-3) / 1e9 / peak, 4)}
+                               for n, k in kernels.items()}}
 
     # ---- end to end: host buffers in, compact cache out, copies inside the timed region ----
     e2e_steps = max(3, min(args.steps, 50))
