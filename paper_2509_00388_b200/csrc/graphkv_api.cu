@@ -277,6 +277,21 @@ graphkv_status launch_ex(const char *name, void (*kern)(KArgs...), dim3 grid, di
     return GRAPHKV_OK;
 }
 
+// Runs `setup` once per device (function attributes are per device); returns its result.
+template <typename F> bool once_per_device(std::mutex &mu, signed char (&state)[64], F setup)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> lk(mu);
+    if (state[dev] == 0) state[dev] = setup() ? 1 : -1;
+    return state[dev] > 0;
+}
+
+template <typename Kern> bool set_smem(Kern k, size_t bytes)
+{
+    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
 // ---- step (I) ------------------------------------------------------------------------------
 // Attention mass before pooling, a [units][N], SIMT path (any dtype).
 template <typename T>
@@ -289,14 +304,12 @@ graphkv_status run_mass_simt(const Dims &d, const Layout &l, const T *Q, const T
                (score_stats_simt<T><<<dim3(l.n_stat_chunks, d.units), threads, 0, st>>>(
                    d, Q, K, part, l.n_stat_chunks, at<int>(ws, l.status))));
     const size_t smem = ((size_t)d.GW * kHeadDim + 2 * d.GW) * sizeof(float);
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[sizeof(T) == 2]) {
-        if (cudaFuncSetAttribute(score_emit_simt<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(((size_t)kMaxRows * kHeadDim + 2 * kMaxRows) * sizeof(float))) !=
-            cudaSuccess)
-            return GRAPHKV_ERR_CUDA;
-        attr_set[sizeof(T) == 2] = true;
-    }
+    static std::mutex mu;
+    static signed char state[64] = {};
+    if (!once_per_device(mu, state, [] {
+            return set_smem(score_emit_simt<T>, ((size_t)kMaxRows * kHeadDim + 2 * kMaxRows) * sizeof(float));
+        }))
+        return GRAPHKV_ERR_CUDA;
     GKV_LAUNCH("score_emit_simt", st,
                (score_emit_simt<T><<<dim3(ceil_div(d.N, kEmitChunk), d.units), kEmitThreads, smem,
                                      st>>>(d, Q, K, part, l.n_stat_chunks, a)));
@@ -342,10 +355,6 @@ bool make_k_tensormap(CUtensorMap *tm, const void *K, const Dims &d, int rows)
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename Kern> bool set_smem(Kern k, size_t bytes)
-{
-    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
-}
 
 // Attention mass before pooling, a [units][N], tensor-core path (bf16).
 graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
@@ -357,14 +366,14 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
     const int rows_pad = 128 * row_tiles;
     const int stages = row_tiles == 1 ? 5 : 4;
     const size_t smem = tc::score_smem_bytes(rows_pad, stages);
-    static std::once_flag once;
-    static bool attr_ok = true;
-    std::call_once(once, [] {
+    static std::mutex mu;
+    static signed char state[64] = {};
+    if (!once_per_device(mu, state, [] {
         const size_t mx = std::max(tc::score_smem_bytes(256, 4), tc::score_smem_bytes(128, 5));
-        attr_ok = set_smem(tc::score_stats_tc<1>, mx) && set_smem(tc::score_stats_tc<2>, mx) &&
+        return set_smem(tc::score_stats_tc<1>, mx) && set_smem(tc::score_stats_tc<2>, mx) &&
                   set_smem(tc::score_emit_tc<1>, mx) && set_smem(tc::score_emit_tc<2>, mx);
-    });
-    if (!attr_ok) return GRAPHKV_ERR_CUDA;
+        }))
+        return GRAPHKV_ERR_CUDA;
     const int tiles_stats = ceil_div(d.L, tc::kTileKeys), tiles_emit = ceil_div(d.N, tc::kTileKeys);
     const int group = units_per_group(d);
     graphkv_status rc = GRAPHKV_OK;
@@ -420,16 +429,16 @@ template <typename Args>
 graphkv_status launch_cluster(const char *name, void (*kern)(Args), Args args, int clusters, int C,
                               size_t smem, cudaStream_t st)
 {
-    static std::once_flag once;
-    static bool attr_ok = true;
-    std::call_once(once, [] {
+    static std::mutex mu;
+    static signed char state[64] = {};
+    if (!once_per_device(mu, state, [] {
         const size_t mx = cs::smem_bytes(cs::kMaxChunk, cs::kMaxHalo);
-        attr_ok = set_smem(cs::pool_select_kernel<1>, mx) && set_smem(cs::pool_select_kernel<2>, mx) &&
+        return set_smem(cs::pool_select_kernel<1>, mx) && set_smem(cs::pool_select_kernel<2>, mx) &&
                   set_smem(cs::pool_select_kernel<4>, mx) && set_smem(cs::pool_select_kernel<8>, mx) &&
                   set_smem(cs::pool_select_kernel<16>, mx) && set_smem(cs::pool_select_kernel<32>, mx) &&
                   set_smem(cs::finish_kernel, mx);
-    });
-    if (!attr_ok) return GRAPHKV_ERR_CUDA;
+        }))
+        return GRAPHKV_ERR_CUDA;
     args.wait_prior = next_launch_is_dependent();
     return launch_ex(name, kern, dim3(clusters * C), dim3(cs::kThreads), smem, st, args.wait_prior != 0, C,
                      args);
@@ -478,14 +487,14 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *
     if (sp.ok) {
         CUtensorMap tmK;
         if (!make_k_tensormap(&tmK, K, d, d.L)) return GRAPHKV_ERR_CUDA;
-        static std::once_flag once;
-        static bool attr_ok = true;
-        std::call_once(once, [] {
-            attr_ok = set_smem(tc::similarity_tc<16>, tc::sim_smem_bytes<16>(5)) &&
+        static std::mutex mu;
+        static signed char state[64] = {};
+        if (!once_per_device(mu, state, [] {
+            return set_smem(tc::similarity_tc<16>, tc::sim_smem_bytes<16>(5)) &&
                       set_smem(tc::similarity_tc<32>, tc::sim_smem_bytes<32>(5)) &&
                       set_smem(tc::similarity_tc<64>, tc::sim_smem_bytes<64>(4));
-        });
-        if (!attr_ok) return GRAPHKV_ERR_CUDA;
+            }))
+            return GRAPHKV_ERR_CUDA;
         const int group = units_per_group(d);
         for (int u0 = 0; u0 < d.units; u0 += group) {
             const int nu = std::min(group, d.units - u0);

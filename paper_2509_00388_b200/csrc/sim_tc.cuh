@@ -292,6 +292,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 if (lane == 0) tau[c] = bstar <= 0 ? -1.0f : (float)bstar * (2.0f / kMaxBins) - 1.0f;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (et == 0) xchg[1] = 0;
             // 2. list the edges that reach the threshold.  theta is the threshold brought to the scale
             //    of dot / |k_j|, lowered by a few ulps so that no edge with cosine >= tau is missed.
             //    Branch-free: a thread's first kSlots edges of a source go to slots of its own by
@@ -384,11 +385,16 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                     if (valid && pos < kCandCap) list[c * kCandCap + pos] = Cand{e, cd.j};
                     total += __popc(bm);
                 }
-                if (lane == 0) cnt[c] = basep + total;
+                if (lane == 0) {
+                    cnt[c] = basep + total;
+                    if (basep + total > kCandCap) xchg[1] = 1;      // some list overflowed
+                }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             // 3. a list that outgrew its capacity: exact m-th largest (edge desc, position asc)
-            for (int c = 0; c < d.K_src; ++c) {
+            const bool any_overflow = xchg[1] != 0;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            for (int c = 0; c < d.K_src && any_overflow; ++c) {
                 if (cnt[c] <= kCandCap) continue;                 // uniform: shared memory value
                 unsigned long long t64 = 0ull;
                 const float sinv = src_inv[c];
