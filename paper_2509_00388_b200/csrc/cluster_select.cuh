@@ -3,7 +3,8 @@
 //
 //   pool_select_kernel   max pooling of the attention mass (step (I), last part) and the
 //                        source nodes of Eq. 2: top-k of the pooled scores.
-//   finish_kernel        the decay rounds of Eq. 5 / Algorithm 2 over the fixed neighbour lists,
+//   finish_kernel        the neighbourhoods of Eq. 3 merged from the per-chunk candidate lists of
+//                        the similarity sweep, the decay rounds of Eq. 5 / Algorithm 2 over them,
 //                        the final k_l selection and the gather of the compact cache.
 //
 // Every exact top-k here is a most-significant-digit radix search over the order-preserving

@@ -7,10 +7,14 @@
 //   score_emit_tc   D = K Q^T  (keys on TMEM lanes): a[j] = sum_r 2^(l2[r][j] - c_r),
 //                   c_r = max_r + log2(Z_r), i.e. the softmax probabilities summed over the
 //                   window rows and grouped heads, one thread per key.
-// The second sweep re-reads K right after the first, so it is served by L2 when a launch's
-// share of K fits there.  Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA
-// issuer and TMEM owner, warps 2..9 = epilogue (two sets of four warps covering the four TMEM
-// lane quadrants; the sets split the accumulator columns).
+// The second sweep re-reads K right after the first, so it is served by L2 as far as the keys
+// fit there.  The statistics CTAs of a unit leave their partial (max, sum) per row in global
+// memory and the last of them to finish (an arrival counter) merges them into c_r.  One
+// exponential in four is evaluated by a cubic on the FMA pipe: at 256 query rows per KV head the
+// MUFU unit, not HBM, is the ceiling of both sweeps.  Warp roles (320 threads): warp 0 = TMA
+// producer (it starts on the key tiles before the dependency wait: keys are an input of the
+// call), warp 1 = MMA issuer and TMEM owner, warps 2..9 = epilogue (two sets of four warps
+// covering the four TMEM lane quadrants; the sets split the accumulator columns).
 #pragma once
 
 #include "tc_common.cuh"

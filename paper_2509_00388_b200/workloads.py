@@ -86,7 +86,7 @@ def _register(cfg: GraphKVConfig) -> GraphKVConfig:
     return cfg
 
 
-# The five workloads of the benchmark definition.  Fields the definition leaves open
+# The five benchmark workloads.  Fields their definition leaves open
 # (pool kernel where not given, decay everywhere, neighbours) take pool_kernel=7,
 # decay=1.0 and the adaptive neighbour rule's value written out explicitly.
 TINY = _register(GraphKVConfig(
