@@ -380,6 +380,7 @@ struct PoolSelectArgs {
     float *s;              // [units][N] scores: written when pooling, read otherwise
     int k;                 // sources to pick (0: none)
     int *src_out;          // [units][k] ascending positions
+    const uint32_t *mass_hist;  // optional [units][kBins]: histogram of values the scores dominate
     uint32_t *zero;        // optional: [units][zero_words] words this launch clears for later kernels
     int zero_words;
     int wait_prior;        // launched with programmatic stream serialization
@@ -387,6 +388,111 @@ struct PoolSelectArgs {
 
 // grid = units * C CTAs in clusters of C; block kThreads.  kPer >= chunk / kThreads: elements of
 // the chunk a thread pools (a power of two up to kMaxPerThread).
+// Top-k of the cluster's row when a histogram of values that the row dominates elementwise is at
+// hand (the pooled scores against the histogram of the attention mass before pooling: pooling only
+// raises values, so the k-th largest pooled score is at least the k-th largest mass).  The highest
+// digit b with k histogram entries in digits >= b therefore bounds the k-th largest row value from
+// below; the row's elements with digit >= b are few (at most pool_kernel times the histogram's
+// count); each CTA lists its own, the first CTA pulls the lists through distributed shared memory
+// and ranks them by counting.  Returns false (in every CTA alike, nothing written) when they exceed kThreads; the
+// caller then runs the radix search.  `mass_hist`: kBins counts of the top 11 bits.
+__device__ bool cluster_topk_bounded(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                     const float *vals, int n_local, int base, int k,
+                                     const uint32_t *mass_hist, int *out)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // digit b: walk the histogram from the top (thread t owns digits kBins-1-2t and kBins-2-2t)
+    const uint32_t c0 = __ldcg(mass_hist + kBins - 1 - 2 * tid), c1 = __ldcg(mass_hist + kBins - 2 - 2 * tid);
+    uint32_t incl = warp_incl_scan(c0 + c1, lane);
+    if (lane == 31) s.wcnt[warp] = incl;
+    if (tid == 0) {
+        s.misc[0] = 0u;          // digit 0 when the histogram holds fewer than k entries
+        s.misc[7] = 0u;          // this CTA's candidate counter
+    }
+    __syncthreads();
+    if (warp == 0) s.wcnt[lane] = warp_incl_scan(s.wcnt[lane], lane);
+    __syncthreads();
+    incl += warp == 0 ? 0u : s.wcnt[warp - 1];
+    const uint32_t before0 = incl - c0 - c1, before1 = before0 + c0;
+    if (before0 < (uint32_t)k && before0 + c0 >= (uint32_t)k) s.misc[0] = kBins - 1 - 2 * tid;
+    else if (before1 < (uint32_t)k && before1 + c1 >= (uint32_t)k) s.misc[0] = kBins - 2 - 2 * tid;
+    __syncthreads();
+    const uint32_t bdigit = s.misc[0];
+    // this CTA's candidates -> its own lists (keys in hist, positions in tot)
+    for (int i0 = 0; i0 < n_local; i0 += kThreads) {
+        const int i = i0 + tid;
+        uint32_t key = 0;
+        bool cand = false;
+        if (i < n_local) {
+            key = float_to_key(vals[i]);
+            cand = (key >> 21) >= bdigit;
+        }
+        const unsigned bm = __ballot_sync(0xffffffffu, cand);
+        if (bm) {
+            uint32_t basep = 0;
+            if (lane == 0) basep = atomicAdd(&s.misc[7], (uint32_t)__popc(bm));
+            basep = __shfl_sync(0xffffffffu, basep, 0);
+            const uint32_t pos = basep + __popc(bm & ((1u << lane) - 1u));
+            if (cand && pos < (uint32_t)kThreads) {
+                s.hist[pos] = key;
+                s.tot[pos] = (uint32_t)(base + i);
+            }
+        }
+    }
+    __syncthreads();
+    if (C > 1) cl.sync();
+    // candidate t of the concatenated lists; every CTA learns the total, the first CTA pulls them
+    uint32_t total = 0;
+    int mine_p = -1, mine_j = 0;
+    for (int p = 0; p < C; ++p) {
+        const uint32_t n_p = C > 1 ? cl.map_shared_rank(s.misc, p)[7] : s.misc[7];
+        if (n_p > (uint32_t)kThreads) total = 0x40000000u;       // a list overflowed
+        if (tid >= (int)total && tid < (int)(total + n_p)) {
+            mine_p = p;
+            mine_j = tid - (int)total;
+        }
+        total += n_p;
+    }
+    if (total > (uint32_t)kThreads || total < (uint32_t)k) {
+        if (C > 1) cl.sync();                              // nobody still reads another CTA's counter
+        return false;
+    }
+    if (rank == 0) {
+        uint32_t key = 0, pos = 0;
+        if (mine_p >= 0) {
+            key = (C > 1 ? cl.map_shared_rank(s.hist, mine_p) : s.hist)[mine_j];
+            pos = (C > 1 ? cl.map_shared_rank(s.tot, mine_p) : s.tot)[mine_j];
+        }
+        __syncthreads();                                   // own list read before it is overwritten
+        uint32_t *ck = s.hist, *ci = s.tot;
+        if (mine_p >= 0) {
+            ck[tid] = key;
+            ci[tid] = pos;
+        }
+        __syncthreads();
+        // a warp per candidate: its rank among all (value descending, position ascending)
+        int *kept = s.st_idx;                              // [k] positions of the kept, unordered
+        if (tid == 0) s.misc[3] = 0u;      // (word 7 may still be read by the other CTAs)
+        __syncthreads();
+        for (int t = warp; t < (int)total; t += kWarps) {
+            const uint32_t kt = ck[t], pt = ci[t];
+            int r = 0;
+            for (int u = lane; u < (int)total; u += 32) r += (ck[u] > kt) || (ck[u] == kt && ci[u] < pt);
+            r = __reduce_add_sync(0xffffffffu, r);
+            if (lane == 0 && r < k) kept[atomicAdd(&s.misc[3], 1u)] = (int)pt;
+        }
+        __syncthreads();
+        // ascending positions: thread t places kept[t] by counting the smaller ones
+        if (tid < k) {
+            const int pt = kept[tid];
+            int o = 0;
+            for (int u = 0; u < k; ++u) o += kept[u] < pt;
+            out[o] = pt;
+        }
+    }
+    return true;
+}
+
 template <int kPer>
 __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs a)
 {
@@ -434,9 +540,14 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
     }
     __syncthreads();
     if (a.k > 0) {
-        const Threshold th = cluster_kth(cl, C, rank, s, vals, n_local, (uint32_t)a.k);
-        cluster_emit_sorted(cl, C, rank, s, vals, n_local, base, th,
-                            a.src_out + (long long)unit * a.k);
+        int *out = a.src_out + (long long)unit * a.k;
+        const bool done = a.mass_hist && a.k <= kThreads &&
+                          cluster_topk_bounded(cl, C, rank, s, vals, n_local, base, a.k,
+                                               a.mass_hist + (long long)unit * kBins, out);
+        if (!done) {
+            const Threshold th = cluster_kth(cl, C, rank, s, vals, n_local, (uint32_t)a.k);
+            cluster_emit_sorted(cl, C, rank, s, vals, n_local, base, th, out);
+        }
     }
     if (C > 1) cl.sync();      // no CTA leaves while its shared memory may still be read
 }

@@ -27,6 +27,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t status;      // int status word (256 bytes reserved)
     size_t arrivals;    // stats CTAs done per unit [units] (directly after the status word)
+    size_t a_hist;      // histogram of the attention mass [units][2048] (directly after the counters)
     size_t row_c;       // softmax row constants [units][GW]
     size_t part;        // softmax row statistics per key chunk
     size_t a;           // attention mass before pooling [units][N]
@@ -151,6 +152,7 @@ Layout layout_of(const Dims &d)
     l.max_parts = l.n_stat_chunks > 148 ? l.n_stat_chunks : 148;
     l.status = take(kAlign);
     l.arrivals = take((size_t)d.units * sizeof(int));
+    l.a_hist = take((size_t)d.units * tc::kMassBins * sizeof(uint32_t));
     l.row_c = take((size_t)d.units * d.GW * sizeof(float));
     l.part = take((size_t)d.units * l.max_parts * d.GW * 2 * sizeof(float));
     l.a = take((size_t)d.units * d.N * sizeof(float));
@@ -382,7 +384,7 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
         const int chunks_s = sweep_chunks(nu, tiles_stats, 1, l.max_parts);
         const int chunks_e = sweep_chunks(nu, tiles_emit, 1, 1 << 20);
         tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), at<float>(ws, l.row_c), at<int>(ws, l.arrivals), a,
-                           at<int>(ws, l.status), u0, chunks_s, tiles_stats, chunks_s, stages, 0};
+                           at<uint32_t>(ws, l.a_hist), at<int>(ws, l.status), u0, chunks_s, tiles_stats, chunks_s, stages, 0};
         tc::ScoreTcArgs ea = sa;
         ea.chunks = chunks_e;
         ea.n_tiles = tiles_emit;
@@ -446,13 +448,15 @@ graphkv_status launch_cluster(const char *name, void (*kern)(Args), Args args, i
 
 // Pooling of a -> s (when a != nullptr) and the k source nodes of Eq. 2 (when k > 0).
 // `zero` (optional): zero_words words per unit cleared on the way, for the kernels that follow.
+// `mass_hist` (optional): per unit, a histogram of values the scores dominate (see the kernel).
 graphkv_status run_pool_sources(const Dims &d, const float *a, float *s, int k, int *src,
-                                uint32_t *zero, int zero_words, cudaStream_t st)
+                                const uint32_t *mass_hist, uint32_t *zero, int zero_words,
+                                cudaStream_t st)
 {
     if (!a && k == 0) return GRAPHKV_OK;
     const ClusterPlan cp = cluster_plan(d);
     if (cp.ok) {
-        cs::PoolSelectArgs pa{d, cp.C, cp.chunk, a ? cp.halo : 0, 0, a, s, k, src, zero, zero_words, 0};
+        cs::PoolSelectArgs pa{d, cp.C, cp.chunk, a ? cp.halo : 0, 0, a, s, k, src, mass_hist, zero, zero_words, 0};
         const char *name = a ? (k ? "pool_select_sources" : "pool_max") : "select_sources";
         const size_t smem = cs::smem_bytes(cp.chunk, pa.halo);
         const int per = ceil_div(cp.chunk, cs::kThreads);
@@ -566,10 +570,10 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, float 
 }
 
 // ---- the calls, typed ---------------------------------------------------------------------------
-// Status word and arrival counters start every scoring call at zero.
+// Status word, arrival counters and the mass histogram start every scoring call at zero.
 inline graphkv_status reset_words(const Dims &d, const Layout &l, void *ws, cudaStream_t st)
 {
-    return cudaMemsetAsync(ws, 0, l.arrivals + (size_t)d.units * sizeof(int), st) == cudaSuccess
+    return cudaMemsetAsync(ws, 0, l.a_hist + (size_t)d.units * tc::kMassBins * sizeof(uint32_t), st) == cudaSuccess
                ? GRAPHKV_OK : GRAPHKV_ERR_CUDA;
 }
 
@@ -581,7 +585,7 @@ graphkv_status do_score(const Dims &d, const Layout &l, const T *Q, const T *K, 
     float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
     graphkv_status rc = run_mass(d, l, Q, K, a, ws, st);
     if (rc != GRAPHKV_OK || d.kp == 1) return rc;
-    return run_pool_sources(d, a, scores, 0, nullptr, nullptr, 0, st);
+    return run_pool_sources(d, a, scores, 0, nullptr, nullptr, nullptr, 0, st);
 }
 
 template <typename T>
@@ -591,7 +595,7 @@ graphkv_status do_propagate(const Dims &d, const Layout &l, const T *K, float *s
     if (d.K_src == 0) return GRAPHKV_OK;
     int *src = src_out ? src_out : at<int>(ws, l.src);
     const bool tc_graph = graph_active(d) && sim_plan(d, sizeof(T) == 2).ok;
-    graphkv_status rc = run_pool_sources(d, nullptr, scores, d.K_src, src,
+    graphkv_status rc = run_pool_sources(d, nullptr, scores, d.K_src, src, nullptr,
                                          tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr,
                                          d.K_src * kCandBins, st);
     if (rc != GRAPHKV_OK || !graph_active(d)) return rc;
@@ -612,7 +616,10 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
     if (rc != GRAPHKV_OK) return rc;
     int *src = at<int>(ws, l.src);
     const bool tc_graph = graph && sim_plan(d, sizeof(T) == 2).ok;
+    // the tensor-core emit sweep leaves a histogram of the attention mass behind
+    const bool have_hist = sizeof(T) == 2 && !env_int("GRAPHKV_FORCE_SIMT", 0);
     rc = run_pool_sources(d, d.kp > 1 ? a : nullptr, s, graph ? d.K_src : 0, src,
+                          have_hist ? at<uint32_t>(ws, l.a_hist) : nullptr,
                           tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr, d.K_src * kCandBins, st);
     if (rc != GRAPHKV_OK) return rc;
     if (graph && (rc = run_graph(d, l, K, src, ws, st)) != GRAPHKV_OK) return rc;

@@ -23,6 +23,7 @@ namespace graphkv {
 namespace tc {
 
 constexpr int kScoreThreads = 320;
+constexpr int kMassBins = 2048;         // histogram of the attention mass: top 11 bits of float_to_key
 constexpr int kEpiWarps = 8;
 
 struct ScoreTcArgs {
@@ -32,6 +33,7 @@ struct ScoreTcArgs {
     float *row_c;       // [units][GW] c_r = max_r + log2(Z_r), written by the last stats CTA of a unit
     int *arrivals;      // [units] stats CTAs done per unit (zero before the launch; reset on the way)
     float *a_out;       // [units][N] attention mass before pooling
+    uint32_t *a_hist;   // optional [units][kMassBins]: counts of a by the top bits of its ordered image
     int *status;        // workspace status word
     int unit0;          // first unit of this launch
     int chunks;         // key chunks (CTAs) per unit
@@ -66,7 +68,8 @@ __device__ __forceinline__ ScoreSmem score_smem_layout(uint8_t *raw, int rows_pa
 __host__ __device__ inline size_t score_smem_bytes(int rows_pad, int stages)
 {
     return 1024 + (size_t)rows_pad * 256 + (size_t)stages * kTileBytes + 8 * 8 * 2 + 2 * 8 * 2 + 16 +
-           8192 + 64;      // 8 KB: the CTA's row statistics / row constants and the exchange buffer
+           8192 + 8192 + 64;   // 8 KB: the CTA's row statistics / row constants and the exchange
+                               // buffer; 8 KB: the emit sweep's histogram of the attention mass
 }
 
 // Q rows of the unit -> K-major swizzled operand (rows >= GW zero-filled).  Threads tid of
@@ -336,6 +339,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     const ScoreSmem s = score_smem_layout(smem_raw, kRowsPad, a.stages, &gen);
     float *row_c = reinterpret_cast<float *>(gen + (s.misc - s.q));      // [kRowsPad]
     float *xchg = row_c + kRowsPad;                                     // [2][128]
+    uint32_t *mass_hist = reinterpret_cast<uint32_t *>(gen + (s.misc - s.q) + 8192);   // [kMassBins]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int unit = a.unit0 + blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
     const int chunk = blockIdx.x;
@@ -355,6 +359,8 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     }
     if (a.wait_prior) pdl_wait();
     pdl_launch_dependents();
+    if (a.a_hist)
+        for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads) mass_hist[i] = 0u;
     // c_r of the unit's rows; padding rows contribute 2^-inf = 0
     for (int r = threadIdx.x; r < kRowsPad; r += kScoreThreads)
         row_c[r] = r < d.GW ? __ldcg(a.row_c + (long long)unit * d.GW + r) : INFINITY;
@@ -423,7 +429,11 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (set == 0 && alive) {
                 const int j = (t0 + i) * kTileKeys + key_lane;
-                if (j < d.N) a_row[j] = acc + xchg[buf * 128 + key_lane];
+                if (j < d.N) {
+                    const float aj = acc + xchg[buf * 128 + key_lane];
+                    a_row[j] = aj;
+                    if (a.a_hist) atomicAdd(&mass_hist[float_to_key(aj) >> 21], 1u);
+                }
             }
         }
         ok = alive;
@@ -436,6 +446,10 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    // this CTA's share of the unit's mass histogram (pooling and source selection start from it)
+    if (a.a_hist)
+        for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads)
+            if (mass_hist[i]) atomicAdd(a.a_hist + (long long)unit * kMassBins + i, mass_hist[i]);
 }
 
 }  // namespace tc
