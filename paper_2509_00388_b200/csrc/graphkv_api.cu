@@ -120,6 +120,22 @@ int sweep_chunks(int units, int tiles, int min_chunks, int max_chunks)
     return best;
 }
 
+// ---- row-wise stages on clusters: which rows fit ----------------------------------------------------
+struct ClusterPlan {
+    bool ok;            // the row fits the cluster kernels
+    int C, chunk, halo;
+};
+
+ClusterPlan cluster_plan(const Dims &d)
+{
+    ClusterPlan p{false, 1, 0, (d.kp - 1) / 2};
+    if (env_int("GRAPHKV_NO_CLUSTER", 0)) return p;
+    while (p.C < cs::kMaxCluster && ceil_div(d.N, p.C) > 4096) p.C *= 2;
+    p.chunk = (ceil_div(d.N, p.C) + 31) & ~31;
+    p.ok = p.chunk <= cs::kMaxChunk && p.halo <= cs::kMaxHalo;
+    return p;
+}
+
 // Tensor-core similarity sweep: usable for bf16 keys, up to 64 sources and 32 neighbours.
 struct SimPlan {
     bool ok;
@@ -134,6 +150,7 @@ SimPlan sim_plan(const Dims &d, bool bf16)
     SimPlan p{false, 16, 1, ceil_div(d.N, tc::kTileKeys), 5};
     if (!bf16 || d.K_src < 1 || d.K_src > 64 || d.m < 1 || d.m > tc::kSimMaxNeighbors) return p;
     if (env_int("GRAPHKV_FORCE_SIMT", 0)) return p;
+    if (!cluster_plan(d).ok) return p;          // its candidate lists are merged by the cluster kernel
     p.NP = d.K_src <= 16 ? 16 : (d.K_src <= 32 ? 32 : 64);
     p.stages = p.NP == 64 ? 4 : 5;
     const int cap = 512 / p.NP;
@@ -412,21 +429,6 @@ inline graphkv_status run_mass(const Dims &d, const Layout &l, const float *Q, c
 }
 
 // ---- row-wise stages on clusters -------------------------------------------------------------
-struct ClusterPlan {
-    bool ok;            // the row fits the cluster kernels
-    int C, chunk, halo;
-};
-
-ClusterPlan cluster_plan(const Dims &d)
-{
-    ClusterPlan p{false, 1, 0, (d.kp - 1) / 2};
-    if (env_int("GRAPHKV_NO_CLUSTER", 0)) return p;
-    while (p.C < cs::kMaxCluster && ceil_div(d.N, p.C) > 4096) p.C *= 2;
-    p.chunk = (ceil_div(d.N, p.C) + 31) & ~31;
-    p.ok = p.chunk <= cs::kMaxChunk && p.halo <= cs::kMaxHalo;
-    return p;
-}
-
 template <typename Args>
 graphkv_status launch_cluster(const char *name, void (*kern)(Args), Args args, int clusters, int C,
                               size_t smem, cudaStream_t st)

@@ -168,6 +168,33 @@ def test_identical_keys_take_the_exact_tie_paths(gk):
         assert np.array_equal(staged["idx"][0, h].numpy(), want_idx)
 
 
+@pytest.mark.parametrize("env", [{"GRAPHKV_NO_CLUSTER": "1"}, {"GRAPHKV_FORCE_SIMT": "1"},
+                                 {"GRAPHKV_NO_CLUSTER": "1", "GRAPHKV_FORCE_SIMT": "1"},
+                                 {"GRAPHKV_L2_GROUP_MB": "1"}])
+def test_fallback_kernels_agree_with_the_oracle(gk, env):
+    # the generic row kernels (rows too long for a cluster), the SIMT sweeps (fp32 inputs, many
+    # sources or neighbours) and several launch groups, forced here on a case the fast path covers
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=4500, budget=300, n_q_heads=8, n_kv_heads=2,
+                    n_clusters=32, neighbors=8, batch=2)
+    old = {k: os.environ.get(k) for k in env}
+    os.environ.update(env)
+    try:
+        check(gk, cfg, strict_overlap=False)
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+
+
+def test_row_longer_than_a_cluster_holds(gk):
+    # N above 8 x 32768: pooling, selections, decay and gather take the generic kernels
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=270000, budget=700, n_q_heads=1, n_kv_heads=1,
+                    window=8, n_clusters=64, topk_nodes=8, neighbors=16)
+    check(gk, cfg, strict_overlap=False)
+
+
 def test_strided_inputs(gk):
     # K and V as views of a [batch, L, heads, D] buffer (token-major, the layout of a fused
     # QKV projection): strides are not those of a dense [b, h, L, D] tensor
