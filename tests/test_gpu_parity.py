@@ -188,6 +188,20 @@ def test_fallback_kernels_agree_with_the_oracle(gk, env):
                 os.environ[k] = v
 
 
+@pytest.mark.parametrize("case", [
+    dict(topk_nodes=40, neighbors=12),                  # source count padded to 64
+    dict(topk_nodes=64, neighbors=32),                  # the largest tensor-core similarity case
+    dict(topk_nodes=65, neighbors=8),                   # one more: generic similarity
+    dict(topk_nodes=12, neighbors=33),                  # neighbours above the candidate-list path
+    dict(topk_nodes=12, neighbors=8, pool_kernel=131),  # pooling halo above the cluster kernel's
+    dict(topk_nodes=3, neighbors=32, rounds=5, decay=0.5),
+])
+def test_regime_boundaries(gk, case):
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=6100, budget=400, n_q_heads=8, n_kv_heads=2,
+                    n_clusters=48, **case)
+    check(gk, cfg, strict_overlap=False)
+
+
 def test_row_longer_than_a_cluster_holds(gk):
     # N above 8 x 32768: pooling, selections, decay and gather take the generic kernels
     cfg = wl.scaled(wl.LLAMA_32K, n_prefix=270000, budget=700, n_q_heads=1, n_kv_heads=1,
