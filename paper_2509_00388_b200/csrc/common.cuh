@@ -21,6 +21,7 @@ struct Dims {
     int B, kp, K_src, m, T;
     float lambda;
     int units;                 // batch * hkv independent (sequence, KV head) problems
+    int bf16;                  // inputs are bf16 (else fp32)
     long long qs[3], ks[3], vs[3];
 };
 

@@ -76,6 +76,7 @@ graphkv_status resolve(const graphkv_params *p, Dims *d)
     d->B = p->budget; d->kp = p->pool_kernel; d->K_src = p->topk_nodes;
     d->m = graphkv_resolve_neighbors(N, p->neighbors);
     d->T = p->rounds; d->lambda = p->decay; d->units = p->batch * p->n_kv_heads;
+    d->bf16 = p->dtype == GRAPHKV_BF16 ? 1 : 0;
     for (int i = 0; i < 3; ++i) {
         d->qs[i] = p->q_stride[i]; d->ks[i] = p->k_stride[i]; d->vs[i] = p->v_stride[i];
     }
@@ -176,10 +177,12 @@ Layout layout_of(const Dims &d)
     l.s = take((size_t)d.units * d.N * sizeof(float));
     l.src = take((size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * sizeof(int));
     const size_t pairs = (size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * (d.m > 0 ? d.m : 1);
-    l.sims = take((size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * d.N * sizeof(float));
+    // the dense edge rows exist only for the generic similarity path
+    const SimPlan sp0 = sim_plan(d, d.bf16 != 0);
+    l.sims = take(sp0.ok ? kAlign : (size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * d.N * sizeof(float));
     l.nbr_idx = take(pairs * sizeof(int));
     l.nbr_e = take(pairs * sizeof(float));
-    const SimPlan sp = sim_plan(d, true);
+    const SimPlan sp = sim_plan(d, d.bf16 != 0);
     const size_t slots = sp.ok ? (size_t)d.units * d.K_src * sp.chunks : 1;
     l.cand = take(slots * kCandCap * sizeof(Cand));
     l.cand_hist = take((size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * kCandBins * sizeof(uint32_t));
@@ -544,7 +547,7 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, float 
     if (cp.ok) {
         cs::FinishArgs fa{d, cp.C, cp.chunk, 0, s, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e),
                           has_graph ? 1 : 0, has_graph && merge ? 1 : 0, at<Cand>(ws, l.cand),
-                          at<uint32_t>(ws, l.cand_hist), sim_plan(d, true).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
+                          at<uint32_t>(ws, l.cand_hist), sim_plan(d, d.bf16 != 0).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
                           static_cast<const unsigned char *>(K), static_cast<const unsigned char *>(V),
                           static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0};
         const char *name = has_graph ? (do_select ? "decay_select_gather" : "decay_rounds") : "select_gather";
