@@ -11,10 +11,12 @@
 // fit there.  The statistics CTAs of a unit leave their partial (max, sum) per row in global
 // memory and the last of them to finish (an arrival counter) merges them into c_r.  One
 // exponential in four is evaluated by a cubic on the FMA pipe: at 256 query rows per KV head the
-// MUFU unit, not HBM, is the ceiling of both sweeps.  Warp roles (320 threads): warp 0 = TMA
-// producer (it starts on the key tiles before the dependency wait: keys are an input of the
-// call), warp 1 = MMA issuer and TMEM owner, warps 2..9 = epilogue (two sets of four warps
-// covering the four TMEM lane quadrants; the sets split the accumulator columns).
+// MUFU unit, not HBM, is the ceiling of both sweeps; the multiply-adds around the exponentials
+// run on packed pairs (fma.rn.f32x2) to halve their issue slots.  Warp roles (576 threads):
+// warp 0 = TMA producer (it starts on the key tiles before the dependency wait: keys are an
+// input of the call), warp 1 = MMA issuer and TMEM owner, warps 2..17 = epilogue (four sets of
+// four warps covering the four TMEM lane quadrants; the sets split the accumulator columns, at
+// most 64 each, copy them to registers and free the TMEM buffer before the arithmetic).
 #pragma once
 
 #include "tc_common.cuh"
@@ -22,9 +24,10 @@
 namespace graphkv {
 namespace tc {
 
-constexpr int kScoreThreads = 320;
+constexpr int kScoreThreads = 576;       // producer warp, MMA warp, 16 epilogue warps
 constexpr int kMassBins = 2048;         // histogram of the attention mass: top 11 bits of float_to_key
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
+constexpr int kScratchBytes = 10240;     // row constants (1 KB) + four exchange buffers of 4 x 128 floats
 
 struct ScoreTcArgs {
     Dims d;
@@ -44,7 +47,7 @@ struct ScoreTcArgs {
 };
 
 struct ScoreSmem {
-    uint32_t q, stage0, full0, empty0, tfull0, tempty0, tmem_slot, misc;
+    uint32_t q, stage0, full0, empty0, tfull0, tempty0, tmem_slot, xbar0, misc;
 };
 
 // Carve dynamic shared memory (1024-byte aligned base): Q operand, K stages, barriers.
@@ -61,15 +64,16 @@ __device__ __forceinline__ ScoreSmem score_smem_layout(uint8_t *raw, int rows_pa
     s.tfull0 = s.empty0 + 8 * 8;
     s.tempty0 = s.tfull0 + 2 * 8;
     s.tmem_slot = s.tempty0 + 2 * 8;
-    s.misc = s.tmem_slot + 16;
+    s.xbar0 = s.tmem_slot + 16;
+    s.misc = s.xbar0 + 4 * 8;
     return s;
 }
 
 __host__ __device__ inline size_t score_smem_bytes(int rows_pad, int stages)
 {
-    return 1024 + (size_t)rows_pad * 256 + (size_t)stages * kTileBytes + 8 * 8 * 2 + 2 * 8 * 2 + 16 +
-           8192 + 8192 + 64;   // 8 KB: the CTA's row statistics / row constants and the exchange
-                               // buffer; 8 KB: the emit sweep's histogram of the attention mass
+    return 1024 + (size_t)rows_pad * 256 + (size_t)stages * kTileBytes + 8 * 8 * 2 + 2 * 8 * 2 + 16 + 4 * 8 +
+           kScratchBytes + 8192 + 64;   // scratch: the CTA's row statistics / row constants and the
+                                        // exchange buffers; 8 KB: the emit sweep's histogram of the mass
 }
 
 // Q rows of the unit -> K-major swizzled operand (rows >= GW zero-filled).  Threads tid of
@@ -111,8 +115,9 @@ __device__ __forceinline__ uint32_t score_setup(const ScoreSmem &s, uint8_t *gen
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(s.tfull0 + 8 * i, 1);
-            mbar_init(s.tempty0 + 8 * i, 8);       // the eight epilogue warps
+            mbar_init(s.tempty0 + 8 * i, kEpiWarps);
         }
+        for (int i = 0; i < 4; ++i) mbar_init(s.xbar0 + 8 * i, kEpiWarps);
         mbar_fence_init();
         tma_prefetch_desc(tmK);
     }
@@ -164,15 +169,8 @@ __device__ __forceinline__ void stats_fold(float (&v)[32], float scale, float &m
     const float mn = fmaxf(mx, cm * scale);
     z *= ex2(mx - mn);
     mx = mn;
-    float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        z0 += ex2(fmaf(v[i], scale, -mn));
-        z1 += ex2(fmaf(v[i + 1], scale, -mn));
-        z2 += ex2(fmaf(v[i + 2], scale, -mn));
-        z3 += ex2_poly3(fmaf(v[i + 3], scale, -mn));      // one exponential in four off the MUFU unit
-    }
-    z += (z0 + z1) + (z2 + z3);
+    const uint64_t nm = pack2(-mn, -mn);
+    z += ex2_sum32(v, pack2(scale, scale), [&](int) { return make_ulonglong2(nm, nm); });
 }
 
 // kRowTiles = 1 (G*W <= 128) or 2 (G*W <= 256).  grid (chunks, units of the launch).
@@ -194,7 +192,8 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     tile_range(a.n_tiles, a.chunks, chunk, &t0, &t1);
     const int n_local = t1 - t0;
 
-    float2 *cta_part = reinterpret_cast<float2 *>(gen + (s.misc - s.q));      // [2][kRowsPad]
+    constexpr int kParts = 4 / kRowTiles;            // epilogue warp sets per row
+    float2 *cta_part = reinterpret_cast<float2 *>(gen + (s.misc - s.q));      // [kParts][kRowsPad]
     int *s_flag = reinterpret_cast<int *>(gen + (s.tmem_slot - s.q)) + 2;
     const int n_ahead = min(n_local, a.stages);
 
@@ -237,49 +236,51 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             }
         }
     } else {
-        // epilogue: thread = query row (TMEM lane), warp set = half of the key columns
+        // epilogue: thread = query row (TMEM lane); the four warp sets split the accumulator's
+        // columns (row tile, then keys).
+        constexpr int kSetCols = kBufCols / 4;             // 32 or 64
         const int quad = warp & 3, set = (warp - 2) >> 2;
         const int row = quad * 32 + lane;
+        const int col0 = set * kSetCols, rt = col0 >> 7, key_off = col0 & 127;
         const float scale = rsqrtf((float)kHeadDim) * kLog2e;
-        float mx[kRowTiles], z[kRowTiles];
-        int lim[kRowTiles];                      // last visible key of the row
-#pragma unroll
-        for (int rt = 0; rt < kRowTiles; ++rt) {
-            mx[rt] = kNegBig;
-            z[rt] = 0.f;
-            const int r = rt * 128 + row;
-            lim[rt] = d.N + (r < d.GW ? r % d.W : 0);
-        }
+        float mx = kNegBig, z = 0.f;
+        const int r = rt * 128 + row;
+        const int lim = d.N + (r < d.GW ? r % d.W : 0);      // last visible key of the row
+        // A thread copies its columns to registers and hands the TMEM buffer back before the
+        // arithmetic, so the next MMA never waits for exponentials.
         bool alive = true;
         for (int i = 0; i < n_local && alive; ++i) {
             const int buf = i & 1, bph = (i >> 1) & 1;
             alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, bph));
             if (!alive) break;
             tc_fence_after();
-            const int key0 = (t0 + i) * kTileKeys + set * 64;
-            const bool masked = key0 + 63 > d.N;          // window keys or the tail past L
+            uint32_t raw[kSetCols / 32][32];
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kBufCols + col0;
 #pragma unroll
-            for (int rt = 0; rt < kRowTiles; ++rt) {
+            for (int c = 0; c < kSetCols / 32; ++c) tmem_ld32_issue(t_row + c * 32, raw[c]);
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    float v[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kBufCols + rt * 128 +
-                                  set * 64 + c * 32, v);
-                    if (masked) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (key0 + c * 32 + e > lim[rt]) v[e] = -INFINITY;
-                    }
-                    stats_fold(v, scale, mx[rt], z[rt]);
-                }
-            }
+            for (int c = 0; c < kSetCols / 32; ++c) tmem_ld_fence(raw[c]);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(s.tempty0 + 8 * buf);
+            const int key0 = (t0 + i) * kTileKeys + key_off;
+            const bool masked = key0 + kSetCols - 1 > d.N;      // window keys or the tail past L
+#pragma unroll
+            for (int c = 0; c < kSetCols / 32; ++c) {
+                float v[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(raw[c][e]);
+                if (masked) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (key0 + c * 32 + e > lim) v[e] = -INFINITY;
+                }
+                stats_fold(v, scale, mx, z);
+            }
         }
         ok = alive;
-#pragma unroll
-        for (int rt = 0; rt < kRowTiles; ++rt) cta_part[set * kRowsPad + rt * 128 + row] = make_float2(mx[rt], z[rt]);
+        // partial p of row r: the sets that share the row's tile
+        cta_part[(set % kParts) * kRowsPad + r] = make_float2(mx, z);
     }
     if (!ok && a.status) atomicExch(a.status, (int)GRAPHKV_ERR_TIMEOUT);
     tc_fence_before();
@@ -292,10 +293,18 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     // this CTA's statistics of each row; the last CTA of the unit to get here merges all chunks
     // into the unit's row constants c_r
     for (int r = threadIdx.x; r < d.GW; r += kScoreThreads) {
-        const float2 p0 = cta_part[r], p1 = cta_part[kRowsPad + r];
-        const float mx = fmaxf(p0.x, p1.x);
+        float2 p[kParts];
+        float mx = kNegBig;
+#pragma unroll
+        for (int k = 0; k < kParts; ++k) {
+            p[k] = cta_part[k * kRowsPad + r];
+            mx = fmaxf(mx, p[k].x);
+        }
+        float z = 0.f;
+#pragma unroll
+        for (int k = 0; k < kParts; ++k) z += p[k].y * ex2(p[k].x - mx);
         reinterpret_cast<float2 *>(a.part)[((long long)unit * a.stats_chunks + chunk) * d.GW + r] =
-            make_float2(mx, p0.y * ex2(p0.x - mx) + p1.y * ex2(p1.x - mx));
+            make_float2(mx, z);
     }
     __threadfence();
     __syncthreads();
@@ -338,8 +347,8 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     uint8_t *gen;
     const ScoreSmem s = score_smem_layout(smem_raw, kRowsPad, a.stages, &gen);
     float *row_c = reinterpret_cast<float *>(gen + (s.misc - s.q));      // [kRowsPad]
-    float *xchg = row_c + kRowsPad;                                     // [2][128]
-    uint32_t *mass_hist = reinterpret_cast<uint32_t *>(gen + (s.misc - s.q) + 8192);   // [kMassBins]
+    float *xchg = row_c + 256;                                          // [4 tiles][4 sets][128]
+    uint32_t *mass_hist = reinterpret_cast<uint32_t *>(gen + (s.misc - s.q) + kScratchBytes);   // [kMassBins]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int unit = a.unit0 + blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
     const int chunk = blockIdx.x;
@@ -361,9 +370,9 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     pdl_launch_dependents();
     if (a.a_hist)
         for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads) mass_hist[i] = 0u;
-    // c_r of the unit's rows; padding rows contribute 2^-inf = 0
+    // -c_r of the unit's rows; padding rows contribute 2^-inf = 0
     for (int r = threadIdx.x; r < kRowsPad; r += kScoreThreads)
-        row_c[r] = r < d.GW ? __ldcg(a.row_c + (long long)unit * d.GW + r) : INFINITY;
+        row_c[r] = r < d.GW ? -__ldcg(a.row_c + (long long)unit * d.GW + r) : -INFINITY;
     __syncthreads();
 
     if (warp == 0) {
@@ -390,50 +399,71 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             }
         }
     } else {
-        // epilogue: thread = key (TMEM lane), warp set = half of the query rows
+        // epilogue: thread = key (TMEM lane); the four warp sets split the query rows (x32 column
+        // slices, at most two each).  A thread copies its slices to registers and hands the TMEM
+        // buffer back before the arithmetic, so the next MMA never waits for exponentials.
         const int quad = warp & 3, set = (warp - 2) >> 2;
         const int key_lane = quad * 32 + lane;
         const float scale = rsqrtf((float)kHeadDim) * kLog2e;
-        const int n_slices = (d.GW + 31) >> 5;                 // x32 column slices in use
-        const int s_begin = set == 0 ? 0 : (n_slices + 1) >> 1;
-        const int s_end = set == 0 ? (n_slices + 1) >> 1 : n_slices;
+        const uint64_t scale2 = pack2(scale, scale);
+        const int n_slices = (d.GW + 31) >> 5;                 // x32 column slices in use (<= 8)
+        const int s_begin = (set * n_slices) >> 2, s_end = ((set + 1) * n_slices) >> 2;
         float *a_row = a.a_out + (long long)unit * d.N;
+        // A thread copies its slices to registers and hands the TMEM buffer back before the
+        // arithmetic, so the next MMA never waits for exponentials.
+        const uint32_t t_set = tmem_base + ((uint32_t)(quad * 32) << 16) + s_begin * 32;
         bool alive = true;
-        for (int i = 0; i < n_local; ++i) {
-            const int buf = i & 1, bph = (i >> 1) & 1;
-            float acc = 0.f;
-            if (alive) alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, bph));
-            if (alive) {
-                tc_fence_after();
-                for (int sl = s_begin; sl < s_end; ++sl) {
-                    float v[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kBufCols + sl * 32, v);
-                    const float4 *c4 = reinterpret_cast<const float4 *>(row_c + sl * 32);
-                    float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
+        auto sum_slice = [&](const uint32_t (&reg)[32], int sl) {
+            float v[32];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float4 c = c4[e];
-                        p0 += ex2(fmaf(v[4 * e], scale, -c.x));
-                        p1 += ex2(fmaf(v[4 * e + 1], scale, -c.y));
-                        p2 += ex2(fmaf(v[4 * e + 2], scale, -c.z));
-                        p3 += ex2_poly3(fmaf(v[4 * e + 3], scale, -c.w));
-                    }
-                    acc += (p0 + p1) + (p2 + p3);
-                }
+            for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(reg[e]);
+            const ulonglong2 *c4 = reinterpret_cast<const ulonglong2 *>(row_c + sl * 32);
+            return ex2_sum32(v, scale2, [&](int q) { return c4[q]; });
+        };
+        for (int i = 0; i < n_local && alive; ++i) {
+            const int buf = i & 1;
+            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, (i >> 1) & 1));
+            if (!alive) break;
+            tc_fence_after();
+            auto release = [&]() {
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(s.tempty0 + 8 * buf);
+            };
+            float acc = 0.f;
+            if (s_end - s_begin == 2) {
+                uint32_t ra[32], rb[32];
+                tmem_ld32_issue(t_set + buf * kBufCols, ra);
+                tmem_ld32_issue(t_set + buf * kBufCols + 32, rb);
+                tmem_ld_fence(ra);
+                tmem_ld_fence(rb);
+                release();
+                acc = sum_slice(ra, s_begin) + sum_slice(rb, s_begin + 1);
+            } else if (s_end - s_begin == 1) {
+                uint32_t ra[32];
+                tmem_ld32_issue(t_set + buf * kBufCols, ra);
+                tmem_ld_fence(ra);
+                release();
+                acc = sum_slice(ra, s_begin);
+            } else {
+                release();
             }
-            // the two sets hold the two halves of each key's row sum
-            if (set == 1) xchg[buf * 128 + key_lane] = acc;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (set == 0 && alive) {
-                const int j = (t0 + i) * kTileKeys + key_lane;
-                if (j < d.N) {
-                    const float aj = acc + xchg[buf * 128 + key_lane];
-                    a_row[j] = aj;
-                    if (a.a_hist) atomicAdd(&mass_hist[float_to_key(aj) >> 21], 1u);
-                }
+            // The sets hold the four parts of each key's row sum.  Each leaves its part in the
+            // exchange buffer of the tile (four in rotation) and arrives on that buffer's
+            // barrier; the sets take turns waiting for all parts, adding them up and storing
+            // the result, so no set waits for another except on its own turn.
+            const int xb = i & 3;
+            xchg[(xb * 4 + set) * 128 + key_lane] = acc;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s.xbar0 + 8 * xb);
+            if (set != xb) continue;
+            alive = __all_sync(0xffffffffu, mbar_wait(s.xbar0 + 8 * xb, (i >> 2) & 1));
+            const int j = (t0 + i) * kTileKeys + key_lane;
+            if (alive && j < d.N) {
+                const float *x = xchg + xb * 512 + key_lane;
+                const float aj = (x[0] + x[128]) + (x[256] + x[384]);
+                a_row[j] = aj;
+                if (a.a_hist) atomicAdd(&mass_hist[float_to_key(aj) >> 21], 1u);
             }
         }
         ok = alive;

@@ -183,6 +183,21 @@ __device__ __forceinline__ float tmem_ld1(uint32_t taddr)
     return __uint_as_float(r);
 }
 
+// Split form of the 32-column load: the registers hold the data only after tmem_ld_fence(r).
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+          "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
 // Split form of the one-column load: issue several, then tmem_ld_fence over their registers.
 __device__ __forceinline__ void tmem_ld1_issue(uint32_t taddr, uint32_t &r)
 {
@@ -216,6 +231,81 @@ __device__ __forceinline__ float ex2_poly3(float x)
     p = fmaf(p, f, 0.693289936f);
     p = fmaf(p, f, 1.0f);
     return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+// Packed pairs of floats in one 64-bit register: sm_100 issues an FMA or an add on both halves as
+// one instruction, which halves the issue slots the exponent arithmetic of the score sweeps takes.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// ex2 of both halves on the MUFU unit
+__device__ __forceinline__ uint64_t ex2_pair(uint64_t x)
+{
+    float lo, hi;
+    unpack2(x, lo, hi);
+    return pack2(ex2(lo), ex2(hi));
+}
+
+// ex2_poly3 of both halves, the float arithmetic on packed pairs (same roundings as ex2_poly3)
+__device__ __forceinline__ uint64_t ex2_poly3_pair(uint64_t x)
+{
+    float lo, hi;
+    unpack2(x, lo, hi);
+    x = pack2(fmaxf(lo, -125.0f), fmaxf(hi, -125.0f));
+    const uint64_t magic = pack2(12582912.0f, 12582912.0f);
+    const uint64_t t = add2(x, magic);
+    const uint64_t n = add2(t, pack2(-12582912.0f, -12582912.0f));
+    const uint64_t f = fma2(n, pack2(-1.0f, -1.0f), x);
+    uint64_t p = fma2(pack2(0.0549740307f, 0.0549740307f), f, pack2(0.242215246f, 0.242215246f));
+    p = fma2(p, f, pack2(0.693289936f, 0.693289936f));
+    p = fma2(p, f, pack2(1.0f, 1.0f));
+    float plo, phi, tlo, thi;
+    unpack2(p, plo, phi);
+    unpack2(t, tlo, thi);
+    return pack2(__int_as_float(__float_as_int(plo) + (__float_as_int(tlo) << 23)),
+                 __int_as_float(__float_as_int(phi) + (__float_as_int(thi) << 23)));
+}
+
+#ifndef GRAPHKV_POLY_PAIRS
+#define GRAPHKV_POLY_PAIRS 1          // of every four pairs, how many take the polynomial
+#endif
+
+// sum over i < 32 of 2^(v[i] * scale + c[i]): nc(q) returns c[4q .. 4q+3] as two packed pairs
+template <class NegC>
+__device__ __forceinline__ float ex2_sum32(const float (&v)[32], uint64_t scale2, NegC nc)
+{
+    uint64_t acc0 = 0ull, acc1 = 0ull;             // (0.f, 0.f)
+#pragma unroll
+    for (int p = 0; p < 16; p += 2) {
+        const ulonglong2 c = nc(p >> 1);
+        const uint64_t x0 = fma2(pack2(v[2 * p], v[2 * p + 1]), scale2, c.x);
+        const uint64_t x1 = fma2(pack2(v[2 * p + 2], v[2 * p + 3]), scale2, c.y);
+        acc0 = add2(acc0, (p & 3) >= 4 - GRAPHKV_POLY_PAIRS ? ex2_poly3_pair(x0) : ex2_pair(x0));
+        acc1 = add2(acc1, ((p + 1) & 3) >= 4 - GRAPHKV_POLY_PAIRS ? ex2_poly3_pair(x1) : ex2_pair(x1));
+    }
+    float lo, hi;
+    unpack2(add2(acc0, acc1), lo, hi);
+    return lo + hi;
 }
 
 // Byte offset of the 16-byte piece `c16` (0..15) of row `r` inside a K-major, 128-byte-swizzled
