@@ -97,8 +97,11 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     float *tau = src_inv + NP;                                                  // [NP] threshold cosine
     int *cnt = reinterpret_cast<int *>(tau + NP);                               // [NP]
     Cand *list = reinterpret_cast<Cand *>(gen + (s_list - base));               // [NP][kCandCap]
-    uint32_t *max_hist = reinterpret_cast<uint32_t *>(gen + (s_stage0 - base)); // [NP][kMaxBins], after the sweep
-    Cand *own = reinterpret_cast<Cand *>(gen + (s_stage0 - base));              // [NP][256][slots], after max_hist
+    // after the sweep the stage memory holds the bins of the maxima and the threads' edge queues
+    // (a key position takes 26 bits there: rows this kernel is given are shorter than 2^18 keys)
+    constexpr int kQueueCap = 32;                                               // edges per thread
+    uint32_t *max_bin = reinterpret_cast<uint32_t *>(gen + (s_stage0 - base));  // [NP / 4][256] bytes = 4 sources
+    uint2 *queue = reinterpret_cast<uint2 *>(max_bin + (NP / 4) * kSimEpiThreads);  // [kQueueCap][256]
     int *xchg = reinterpret_cast<int *>(gen + (s_tmem - base)) + 2;             // 2 words
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -110,6 +113,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     const __nv_bfloat16 *Kh = a.K + b * d.ks[0] + (long long)h * d.ks[1];
     const int *src = a.src + (long long)unit * d.K_src;
 
+    int n_ahead = 0;                 // tiles thread 0 has requested before the roles split
     if (threadIdx.x == 0) {
         for (int i = 0; i < a.stages; ++i) {
             mbar_init(s_full0 + 8 * i, 1);
@@ -118,6 +122,15 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         for (int i = 0; i < kSimMaxTiles; ++i) mbar_init(s_done0 + 8 * i, 1);
         mbar_fence_init();
         tma_prefetch_desc(&tmK);
+        // the first ring-full of key tiles is under way while the sources are gathered (keys are an
+        // input of the call: no wait for the kernels before)
+        n_ahead = min(a.stages, n_local);
+        for (int i = 0; i < n_ahead; ++i) {
+            const uint32_t dst = s_stage0 + i * kTileBytes;
+            mbar_expect_tx(s_full0 + 8 * i, kTileBytes);
+            tma_load_4d(dst, &tmK, s_full0 + 8 * i, 0, (t0 + i) * kTileKeys, h, b);
+            tma_load_4d(dst + kHalfBytes, &tmK, s_full0 + 8 * i, 64, (t0 + i) * kTileKeys, h, b);
+        }
     }
     if (warp == 1) {
         tmem_alloc(s_tmem, 512);
@@ -163,8 +176,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
 
     if (warp == 0) {
         if (lane == 0) {
-            int issued = 0;
-            for (int i = 0; i < n_local; ++i) {
+            int issued = n_ahead;
+            for (int i = n_ahead; i < n_local; ++i) {
                 const int st = i % a.stages, ph = (i / a.stages) & 1;
                 if (!mbar_wait(s_empty0 + 8 * st, ph ^ 1)) { ok = false; break; }
                 const uint32_t dst = s_stage0 + st * kTileBytes;
@@ -247,147 +260,117 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         asm volatile("bar.sync 1, 256;" ::: "memory");
         const bool all_alive = xchg[0] != 0;
         if (all_alive) {
+            if (et == 0) xchg[1] = 0;
             // 1. thresholds.  The cosine of a thread's best key for source c is the rounded product
-            //    of its best dot / |k_j| with 1 / |k_c| (rounding is monotone); histogram those over
-            //    [-1, 1] and take the lower edge of the highest bin with m+1 maxima in or above it.
-            for (int i = et; i < d.K_src * kMaxBins; i += kSimEpiThreads) max_hist[i] = 0u;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            //    of its best dot / |k_j| with 1 / |k_c| (rounding is monotone).  Every thread leaves
+            //    the cosine bins (of kMaxBins over [-1, 1]) of its maxima, four sources to a word; a
+            //    warp takes four sources and finds for each, by bisection over the bin index, the
+            //    highest bin with m+1 maxima in or above it; tau is that bin's lower edge.
+            //    (A thread without keys counts in bin 0, which only matters when tau is -1 anyway.)
 #pragma unroll
-            for (int c = 0; c < NP; ++c) {
-                if (c < d.K_src && best[c] > -INFINITY) {
-                    const float e = fminf(fmaxf(best[c] * src_inv[c], -1.0f), 1.0f);
-                    const int bin = min(max(static_cast<int>((e + 1.0f) * (kMaxBins / 2)), 0), kMaxBins - 1);
-                    atomicAdd(&max_hist[c * kMaxBins + bin], 1u);
+            for (int g = 0; g < NP / 4; ++g) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int c = g * 4 + q;
+                    int bin = 0;
+                    if (c < d.K_src && best[c] > -INFINITY) {
+                        const float e = fminf(fmaxf(best[c] * src_inv[c], -1.0f), 1.0f);
+                        bin = min(max(static_cast<int>((e + 1.0f) * (kMaxBins / 2)), 0), kMaxBins - 1);
+                    }
+                    word |= (uint32_t)bin << (8 * q);
                 }
+                max_bin[g * kSimEpiThreads + et] = word;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             const int ew = warp - 2;
-            for (int c = ew; c < d.K_src; c += 8) {
-                constexpr int kPer = kMaxBins / 32;          // lane l holds bins [l * kPer, (l + 1) * kPer)
-                uint32_t hb[kPer], mine = 0;
-#pragma unroll
-                for (int q = 0; q < kPer; ++q) {
-                    hb[q] = max_hist[c * kMaxBins + lane * kPer + q];
-                    mine += hb[q];
-                }
-                uint32_t above = 0;                          // maxima in the lanes above this one
+            for (int g = ew; g * 4 < d.K_src; g += 8) {
+                uint32_t w8[8];              // this lane's eight threads' bins of sources 4g .. 4g+3
                 {
-                    uint32_t incl = mine;              // suffix sum over lanes, log steps
+                    const uint4 lo = *reinterpret_cast<const uint4 *>(max_bin + g * kSimEpiThreads + lane * 8);
+                    const uint4 hi = *reinterpret_cast<const uint4 *>(max_bin + g * kSimEpiThreads + lane * 8 + 4);
+                    w8[0] = lo.x; w8[1] = lo.y; w8[2] = lo.z; w8[3] = lo.w;
+                    w8[4] = hi.x; w8[5] = hi.y; w8[6] = hi.z; w8[7] = hi.w;
+                }
+                uint32_t bstar[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const uint32_t t = __shfl_down_sync(0xffffffffu, incl, o);
-                        if (lane + o < 32) incl += t;
+                for (int bit = 7; bit >= 0; --bit) {
+                    int n[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t cand = bstar[q] | (1u << bit);
+                        n[q] = 0;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) n[q] += ((w8[k] >> (8 * q)) & 0xffu) >= cand ? 1 : 0;
                     }
-                    above = incl - mine;
-                }
-                int bstar = -1;
-                uint32_t run = above;
 #pragma unroll
-                for (int q = kPer - 1; q >= 0; --q) {
-                    run += hb[q];
-                    if (bstar < 0 && run >= (uint32_t)(d.m + 1)) bstar = lane * kPer + q;
-                }
+                    for (int q = 0; q < 4; ++q) n[q] = __reduce_add_sync(0xffffffffu, n[q]);
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) bstar = max(bstar, __shfl_xor_sync(0xffffffffu, bstar, o));
-                if (lane == 0) tau[c] = bstar <= 0 ? -1.0f : (float)bstar * (2.0f / kMaxBins) - 1.0f;
+                    for (int q = 0; q < 4; ++q)
+                        if (n[q] >= d.m + 1) bstar[q] |= 1u << bit;
+                }
+                if (lane < 4 && g * 4 + lane < d.K_src) {
+                    const uint32_t bs = lane == 0 ? bstar[0] : lane == 1 ? bstar[1] : lane == 2 ? bstar[2] : bstar[3];
+                    tau[g * 4 + lane] = bs == 0 ? -1.0f : (float)bs * (2.0f / kMaxBins) - 1.0f;
+                }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (et == 0) xchg[1] = 0;
             // 2. list the edges that reach the threshold.  theta is the threshold brought to the scale
             //    of dot / |k_j|, lowered by a few ulps so that no edge with cosine >= tau is missed.
-            //    Branch-free: a thread's first kSlots edges of a source go to slots of its own by
-            //    predicated stores (2-bit counters packed in registers); only threads with more
-            //    edges of one source than that come back for them below.
-            constexpr int kSlots = NP <= 32 ? 2 : 1;
+            //    Straight-line code: a thread appends the few edges of its keys that pass, as
+            //    (value, source and key), to a queue of its own; afterwards it turns each into a
+            //    cosine, checks it against tau itself and adds it to the source's list (the order
+            //    within a list carries no meaning).  A queue that fills up sends every source of the
+            //    chunk down the exact path of step 3.
             float theta[NP];
 #pragma unroll
             for (int c = 0; c < NP; ++c) {
                 const float q = c < d.K_src ? tau[c] / src_inv[c] : INFINITY;
                 theta[c] = q - fabsf(q) * 2.4e-7f - 1e-30f;
             }
-            uint32_t nfound[NP / 16];                  // 2 bits per source: edges found, saturating at 3
-#pragma unroll
-            for (int w = 0; w < NP / 16; ++w) nfound[w] = 0u;
+            // (branch-free, the store and the count under one predicate; a key past the end of the
+            // row gets a NaN factor, which fails every comparison)
+            uint2 *const q0 = queue + et;
+            const uint32_t q_first = smem_u32(q0), q_step = kSimEpiThreads * sizeof(uint2);
+            const uint32_t q_last = q_first + (kQueueCap - 1) * q_step;
+            uint32_t qa = q_first;
             for (int i = set; i < n_local; i += 2) {
                 const int j = (t0 + i) * kTileKeys + key_lane;
-                const float inv = j < d.N ? inv_norm[i * 128 + key_lane] : 0.f;
+                const float inv = j < d.N ? inv_norm[i * 128 + key_lane] : __int_as_float(0x7fc00000);
                 float v[NP];
                 tmem_ld_np<NP>(lane_addr + i * NP, v);
 #pragma unroll
                 for (int c = 0; c < NP; ++c) {
-                    const float t = v[c] * inv;
-                    const uint32_t n = (nfound[c / 16] >> (2 * (c % 16))) & 3u;
-                    const bool pass = j < d.N && t >= theta[c];
-                    if (pass && n < kSlots) own[(c * kSimEpiThreads + et) * kSlots + n] = Cand{t, j};
-                    if (pass && n < 3u) nfound[c / 16] += 1u << (2 * (c % 16));
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t.reg .u32 a;\n\t"
+                        "setp.ge.f32 p, %1, %3;\n\t"
+                        "min.u32 a, %0, %4;\n\t"
+                        "@p st.shared.v2.b32 [a], {%1, %2};\n\t"
+                        "@p add.u32 %0, %0, %5;\n\t}"
+                        : "+r"(qa)
+                        : "f"(v[c] * inv), "r"(((uint32_t)c << 26) | (uint32_t)j), "f"(theta[c]), "r"(q_last),
+                          "r"(q_step)
+                        : "memory");
                 }
             }
-            uint32_t over = 0;                         // sources of which this thread has more edges
-#pragma unroll
-            for (int c = 0; c < NP; ++c) {
-                const uint32_t n = (nfound[c / 16] >> (2 * (c % 16))) & 3u;
-#pragma unroll
-                for (int q = 0; q < kSlots; ++q)
-                    if (c < d.K_src && n <= (uint32_t)q) own[(c * kSimEpiThreads + et) * kSlots + q] = Cand{0.f, -1};
-                if (c < 32 && n > (uint32_t)kSlots) over |= 1u << (c & 31);
-                if (NP > 32 && c >= 32 && n > (uint32_t)kSlots) over |= 1u << (c & 31);   // approximate: see below
-            }
-            // the rare threads with more edges of a source than slots: rescan that source's column and
-            // append all but the first kSlots through the shared counter
-            uint32_t any_over = over;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) any_over |= __shfl_xor_sync(0xffffffffu, any_over, o);
-            for (int c = 0; c < d.K_src && any_over; ++c) {
-                if (!((any_over >> (c & 31)) & 1u)) continue;
-                const float sinv = src_inv[c];
-                const float q = tau[c] / sinv;
-                const float th = q - fabsf(q) * 2.4e-7f - 1e-30f;
-                const bool mine = (over >> (c & 31)) & 1u;
-                int skip = kSlots;
-                for (int i = set; i < n_local; i += 2) {
-                    const int j = (t0 + i) * kTileKeys + key_lane;
-                    const float t = tmem_ld1(lane_addr + i * NP + c) * (j < d.N ? inv_norm[i * 128 + key_lane] : 0.f);
-                    if (mine && j < d.N && t >= th) {
-                        if (skip > 0) --skip;
-                        else {
-                            const int pos = atomicAdd(&cnt[c], 1);
-                            if (pos < kCandCap) list[c * kCandCap + pos] = Cand{t, j};
-                        }
-                    }
+            const int n_queued = static_cast<int>((qa - q_first) / q_step);
+            if (n_queued > kQueueCap) xchg[1] = 1;                    // entries were lost
+            for (int k = 0; k < min(n_queued, kQueueCap); ++k) {
+                const uint2 en = q0[k * kSimEpiThreads];
+                const int c = en.y >> 26, j = en.y & 0x3ffffffu;
+                const float e = fminf(fmaxf(__uint_as_float(en.x) * src_inv[c], -1.0f), 1.0f);
+                if (e >= tau[c] && j != src_pos[c]) {
+                    const int pos = atomicAdd(&cnt[c], 1);
+                    if (pos < kCandCap) list[c * kCandCap + pos] = Cand{e, j};
                 }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            // gather the threads' own slots into the lists, now as cosines: warp w takes sources
-            // w, w + 8, ...; entries the counter path added before are converted in place first
-            for (int c = ew; c < d.K_src; c += 8) {
-                const int self = src_pos[c];
-                const float sinv = src_inv[c], tc = tau[c];
-                const int n_pre = min(cnt[c], kCandCap);
-                __syncwarp();
-                for (int i = lane; i < n_pre; i += 32) {
-                    Cand cd = list[c * kCandCap + i];
-                    cd.e = fminf(fmaxf(cd.e * sinv, -1.0f), 1.0f);
-                    if (cd.e < tc || cd.j == self) cd.e = kCandEmpty;     // dropped later as empty
-                    list[c * kCandCap + i] = cd;
-                }
-                __syncwarp();
-                int basep = cnt[c];
-                __syncwarp();
-                constexpr int kPerLane = kSimEpiThreads * kSlots / 32;
-                int total = 0;
-#pragma unroll 4
-                for (int q = 0; q < kPerLane; ++q) {
-                    Cand cd = own[c * kSimEpiThreads * kSlots + q * 32 + lane];
-                    const float e = fminf(fmaxf(cd.e * sinv, -1.0f), 1.0f);
-                    const bool valid = cd.j >= 0 && cd.j != self && e >= tc;
-                    const unsigned bm = __ballot_sync(0xffffffffu, valid);
-                    const int pos = basep + total + __popc(bm & ((1u << lane) - 1u));
-                    if (valid && pos < kCandCap) list[c * kCandCap + pos] = Cand{e, cd.j};
-                    total += __popc(bm);
-                }
-                if (lane == 0) {
-                    cnt[c] = basep + total;
-                    if (basep + total > kCandCap) xchg[1] = 1;      // some list overflowed
+            {
+                const bool lost = xchg[1] != 0;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                for (int c = et; c < d.K_src; c += kSimEpiThreads) {
+                    if (lost) cnt[c] = kCandCap + 1;
+                    if (cnt[c] > kCandCap) xchg[1] = 1;               // some list overflowed
                 }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -429,17 +412,15 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 asm volatile("bar.sync 1, 256;" ::: "memory");
             }
             // write the lists out (unused slots marked empty) and count the listed edges per bin
-            for (int c = 0; c < d.K_src; ++c) {
+            for (int idx = et; idx < d.K_src * kCandCap; idx += kSimEpiThreads) {
+                const int c = idx / kCandCap, q = idx % kCandCap;
                 const long long slot = ((long long)unit * d.K_src + c) * a.chunks + chunk;
-                const int n = min(cnt[c], kCandCap);
-                if (et < kCandCap) {
-                    Cand cd{kCandEmpty, -1};
-                    if (et < n) {
-                        cd = list[c * kCandCap + et];
-                        atomicAdd(a.cand_hist + ((long long)unit * d.K_src + c) * kCandBins + cand_bin(cd.e), 1u);
-                    }
-                    a.cand[slot * kCandCap + et] = cd;
+                Cand cd{kCandEmpty, -1};
+                if (q < min(cnt[c], kCandCap)) {
+                    cd = list[c * kCandCap + q];
+                    atomicAdd(a.cand_hist + ((long long)unit * d.K_src + c) * kCandBins + cand_bin(cd.e), 1u);
                 }
+                a.cand[slot * kCandCap + q] = cd;
             }
         } else {
             // a wait ran out: publish empty lists so the merge reads nothing undefined
