@@ -15,8 +15,10 @@
 // run on packed pairs (fma.rn.f32x2) to halve their issue slots.  Warp roles (576 threads):
 // warp 0 = TMA producer (it starts on the key tiles before the dependency wait: keys are an
 // input of the call), warp 1 = MMA issuer and TMEM owner, warps 2..17 = epilogue (four sets of
-// four warps covering the four TMEM lane quadrants; the sets split the accumulator columns, at
-// most 64 each, copy them to registers and free the TMEM buffer before the arithmetic).
+// four warps covering the four TMEM lane quadrants; a thread takes at most 64 accumulator
+// columns of a tile, copies them to registers and frees the TMEM buffer before the arithmetic.
+// At 256 query rows all four sets share each tile and two buffers alternate; at 128 or fewer two
+// sets share a tile, the two pairs take alternate tiles and four buffers rotate).
 #pragma once
 
 #include "tc_common.cuh"
@@ -62,16 +64,16 @@ __device__ __forceinline__ ScoreSmem score_smem_layout(uint8_t *raw, int rows_pa
     s.full0 = s.stage0 + stages * kTileBytes;
     s.empty0 = s.full0 + 8 * 8;
     s.tfull0 = s.empty0 + 8 * 8;
-    s.tempty0 = s.tfull0 + 2 * 8;
-    s.tmem_slot = s.tempty0 + 2 * 8;
+    s.tempty0 = s.tfull0 + 4 * 8;
+    s.tmem_slot = s.tempty0 + 4 * 8;
     s.xbar0 = s.tmem_slot + 16;
-    s.misc = s.xbar0 + 4 * 8;
+    s.misc = s.xbar0 + 8 * 8;
     return s;
 }
 
 __host__ __device__ inline size_t score_smem_bytes(int rows_pad, int stages)
 {
-    return 1024 + (size_t)rows_pad * 256 + (size_t)stages * kTileBytes + 8 * 8 * 2 + 2 * 8 * 2 + 16 + 4 * 8 +
+    return 1024 + (size_t)rows_pad * 256 + (size_t)stages * kTileBytes + 8 * 8 * 2 + 4 * 8 * 2 + 16 + 8 * 8 +
            kScratchBytes + 8192 + 64;   // scratch: the CTA's row statistics / row constants and the
                                         // exchange buffers; 8 KB: the emit sweep's histogram of the mass
 }
@@ -106,18 +108,18 @@ __device__ __forceinline__ void stage_q(uint8_t *q_gen, int rows_pad, const Dims
 // Barriers and TMEM of both sweeps, then the CTA synchronised so that every warp may use them.
 // Returns the TMEM base address.
 __device__ __forceinline__ uint32_t score_setup(const ScoreSmem &s, uint8_t *gen, const CUtensorMap *tmK,
-                                                int stages, uint32_t tmem_cols)
+                                                int stages, uint32_t tmem_cols, int tile_warps)
 {
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
             mbar_init(s.full0 + 8 * i, 1);
             mbar_init(s.empty0 + 8 * i, 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 4; ++i) {
             mbar_init(s.tfull0 + 8 * i, 1);
-            mbar_init(s.tempty0 + 8 * i, kEpiWarps);
+            mbar_init(s.tempty0 + 8 * i, tile_warps);      // the epilogue warps that work on one tile
         }
-        for (int i = 0; i < 4; ++i) mbar_init(s.xbar0 + 8 * i, kEpiWarps);
+        for (int i = 0; i < 8; ++i) mbar_init(s.xbar0 + 8 * i, tile_warps);
         mbar_fence_init();
         tma_prefetch_desc(tmK);
     }
@@ -181,7 +183,11 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     extern __shared__ uint8_t smem_raw[];
     constexpr int kRowsPad = 128 * kRowTiles;
     constexpr int kBufCols = 128 * kRowTiles;        // TMEM columns per accumulator buffer
-    constexpr uint32_t kTmemCols = 2 * kBufCols;
+    constexpr uint32_t kTmemCols = 512;
+    // Every epilogue thread takes 64 accumulator columns of a tile.  With two row tiles the 16
+    // warps share each tile (two buffers); with one, two groups of 8 warps take alternate tiles
+    // (four buffers), so that a round of waiting, loading and releasing covers as much arithmetic.
+    constexpr int kBufs = 512 / kBufCols, kGroups = 2 / kRowTiles;
     const Dims &d = a.d;
     uint8_t *gen;
     const ScoreSmem s = score_smem_layout(smem_raw, kRowsPad, a.stages, &gen);
@@ -192,12 +198,12 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     tile_range(a.n_tiles, a.chunks, chunk, &t0, &t1);
     const int n_local = t1 - t0;
 
-    constexpr int kParts = 4 / kRowTiles;            // epilogue warp sets per row
+    constexpr int kParts = 4 / kRowTiles;            // partial statistics per row
     float2 *cta_part = reinterpret_cast<float2 *>(gen + (s.misc - s.q));      // [kParts][kRowsPad]
     int *s_flag = reinterpret_cast<int *>(gen + (s.tmem_slot - s.q)) + 2;
     const int n_ahead = min(n_local, a.stages);
 
-    const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols);
+    const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols, kEpiWarps / kGroups);
     bool ok = true;
     if (warp == 0) {
         if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b);
@@ -216,7 +222,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
             for (int i = 0; i < n_local; ++i) {
                 const int st = i % a.stages, ph = (i / a.stages) & 1;
-                const int buf = i & 1, bph = (i >> 1) & 1;
+                const int buf = i % kBufs, bph = (i / kBufs) & 1;
                 if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1)) { ok = false; break; }
                 if (!mbar_wait(s.full0 + 8 * st, ph)) { ok = false; break; }
                 tc_fence_after();
@@ -238,10 +244,11 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     } else {
         // epilogue: thread = query row (TMEM lane); the four warp sets split the accumulator's
         // columns (row tile, then keys).
-        constexpr int kSetCols = kBufCols / 4;             // 32 or 64
+        constexpr int kSetCols = 64;
         const int quad = warp & 3, set = (warp - 2) >> 2;
+        const int grp = set / (4 / kGroups);               // tiles grp, grp + kGroups, ...
         const int row = quad * 32 + lane;
-        const int col0 = set * kSetCols, rt = col0 >> 7, key_off = col0 & 127;
+        const int col0 = (set % (4 / kGroups)) * kSetCols, rt = col0 >> 7, key_off = col0 & 127;
         const float scale = rsqrtf((float)kHeadDim) * kLog2e;
         float mx = kNegBig, z = 0.f;
         const int r = rt * 128 + row;
@@ -249,8 +256,8 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         // A thread copies its columns to registers and hands the TMEM buffer back before the
         // arithmetic, so the next MMA never waits for exponentials.
         bool alive = true;
-        for (int i = 0; i < n_local && alive; ++i) {
-            const int buf = i & 1, bph = (i >> 1) & 1;
+        for (int i = grp; i < n_local && alive; i += kGroups) {
+            const int buf = i % kBufs, bph = (i / kBufs) & 1;
             alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, bph));
             if (!alive) break;
             tc_fence_after();
@@ -279,8 +286,8 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             }
         }
         ok = alive;
-        // partial p of row r: the sets that share the row's tile
-        cta_part[(set % kParts) * kRowsPad + r] = make_float2(mx, z);
+        // partial p of row r: the sets (of every group) that hold columns of the row's tile
+        cta_part[(kRowTiles == 1 ? set : set & 1) * kRowsPad + r] = make_float2(mx, z);
     }
     if (!ok && a.status) atomicExch(a.status, (int)GRAPHKV_ERR_TIMEOUT);
     tc_fence_before();
@@ -342,12 +349,18 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     extern __shared__ uint8_t smem_raw[];
     constexpr int kRowsPad = 128 * kColTiles;        // rows of the Q operand (UMMA N)
     constexpr int kBufCols = 128 * kColTiles;
-    constexpr uint32_t kTmemCols = 2 * kBufCols;
+    constexpr uint32_t kTmemCols = 512;
+    // Every epilogue thread takes up to 64 accumulator columns of a tile.  With two column tiles
+    // the 16 warps share each tile (two buffers); with one, two groups of 8 warps take alternate
+    // tiles (four buffers), so that a round of waiting, loading and releasing covers as much
+    // arithmetic.
+    constexpr int kBufs = 512 / kBufCols, kGroups = 2 / kColTiles, kSets = 4 / kGroups;
+    constexpr int kXchg = 16 / kSets;                // exchange buffers in rotation
     const Dims &d = a.d;
     uint8_t *gen;
     const ScoreSmem s = score_smem_layout(smem_raw, kRowsPad, a.stages, &gen);
     float *row_c = reinterpret_cast<float *>(gen + (s.misc - s.q));      // [kRowsPad]
-    float *xchg = row_c + 256;                                          // [4 tiles][4 sets][128]
+    float *xchg = row_c + 256;                                          // [kXchg tiles][kSets][128]
     uint32_t *mass_hist = reinterpret_cast<uint32_t *>(gen + (s.misc - s.q) + kScratchBytes);   // [kMassBins]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int unit = a.unit0 + blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
@@ -358,7 +371,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     const int n_cols = (d.GW + 31) & ~31;            // UMMA N: every x32 slice read below is written
 
     const int n_ahead = min(n_local, a.stages);
-    const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols);
+    const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols, kEpiWarps / kGroups);
     bool ok = true;
     if (warp == 0) {
         if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b);
@@ -382,7 +395,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             const uint32_t idesc = umma_idesc_bf16(128, n_cols);
             for (int i = 0; i < n_local; ++i) {
                 const int st = i % a.stages, ph = (i / a.stages) & 1;
-                const int buf = i & 1, bph = (i >> 1) & 1;
+                const int buf = i % kBufs, bph = (i / kBufs) & 1;
                 if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1)) { ok = false; break; }
                 if (!mbar_wait(s.full0 + 8 * st, ph)) { ok = false; break; }
                 tc_fence_after();
@@ -399,15 +412,15 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             }
         }
     } else {
-        // epilogue: thread = key (TMEM lane); the four warp sets split the query rows (x32 column
-        // slices, at most two each).  A thread copies its slices to registers and hands the TMEM
-        // buffer back before the arithmetic, so the next MMA never waits for exponentials.
+        // epilogue: thread = key (TMEM lane); the warp sets of a tile split the query rows (x32
+        // column slices, at most two each).
         const int quad = warp & 3, set = (warp - 2) >> 2;
+        const int grp = set / kSets, part = set % kSets;       // tiles grp, grp + kGroups, ...
         const int key_lane = quad * 32 + lane;
         const float scale = rsqrtf((float)kHeadDim) * kLog2e;
         const uint64_t scale2 = pack2(scale, scale);
         const int n_slices = (d.GW + 31) >> 5;                 // x32 column slices in use (<= 8)
-        const int s_begin = (set * n_slices) >> 2, s_end = ((set + 1) * n_slices) >> 2;
+        const int s_begin = (part * n_slices) / kSets, s_end = ((part + 1) * n_slices) / kSets;
         float *a_row = a.a_out + (long long)unit * d.N;
         // A thread copies its slices to registers and hands the TMEM buffer back before the
         // arithmetic, so the next MMA never waits for exponentials.
@@ -420,9 +433,9 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             const ulonglong2 *c4 = reinterpret_cast<const ulonglong2 *>(row_c + sl * 32);
             return ex2_sum32(v, scale2, [&](int q) { return c4[q]; });
         };
-        for (int i = 0; i < n_local && alive; ++i) {
-            const int buf = i & 1;
-            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, (i >> 1) & 1));
+        for (int i = grp; i < n_local && alive; i += kGroups) {
+            const int buf = i % kBufs;
+            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, (i / kBufs) & 1));
             if (!alive) break;
             tc_fence_after();
             auto release = [&]() {
@@ -448,20 +461,21 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             } else {
                 release();
             }
-            // The sets hold the four parts of each key's row sum.  Each leaves its part in the
-            // exchange buffer of the tile (four in rotation) and arrives on that buffer's
-            // barrier; the sets take turns waiting for all parts, adding them up and storing
-            // the result, so no set waits for another except on its own turn.
-            const int xb = i & 3;
-            xchg[(xb * 4 + set) * 128 + key_lane] = acc;
+            // The sets of the tile hold the parts of each key's row sum.  Each leaves its part in
+            // the exchange buffer of the tile (kXchg in rotation: a buffer comes round again only
+            // after every warp has left the tile that used it) and arrives on that buffer's
+            // barrier; the sets take turns waiting for all parts, adding them up and storing the
+            // result, so no set waits for another except on its own turn.
+            const int xb = i % kXchg;
+            xchg[(xb * kSets + part) * 128 + key_lane] = acc;
             __syncwarp();
             if (lane == 0) mbar_arrive(s.xbar0 + 8 * xb);
-            if (set != xb) continue;
-            alive = __all_sync(0xffffffffu, mbar_wait(s.xbar0 + 8 * xb, (i >> 2) & 1));
+            if (part != (i / kGroups) % kSets) continue;
+            alive = __all_sync(0xffffffffu, mbar_wait(s.xbar0 + 8 * xb, (i / kXchg) & 1));
             const int j = (t0 + i) * kTileKeys + key_lane;
             if (alive && j < d.N) {
-                const float *x = xchg + xb * 512 + key_lane;
-                const float aj = (x[0] + x[128]) + (x[256] + x[384]);
+                const float *x = xchg + xb * kSets * 128 + key_lane;
+                const float aj = kSets == 4 ? (x[0] + x[128]) + (x[256] + x[384]) : x[0] + x[128];
                 a_row[j] = aj;
                 if (a.a_hist) atomicAdd(&mass_hist[float_to_key(aj) >> 21], 1u);
             }
