@@ -89,6 +89,10 @@ SMALL = [
     dict(n_prefix=3000, budget=500, n_q_heads=8, n_kv_heads=2, window=64, topk_nodes=32, rounds=4),
     dict(n_prefix=2049, budget=100, n_q_heads=4, n_kv_heads=1, window=17, batch=3, neighbors=3),
     dict(n_prefix=1024, budget=1024, n_q_heads=2, n_kv_heads=2, window=8),
+    # query rows per KV head that fill 5, 6 and 7 of the 8 accumulator slices of the score sweeps
+    dict(n_prefix=3500, budget=200, n_q_heads=6, n_kv_heads=2, window=48),
+    dict(n_prefix=2700, budget=150, n_q_heads=5, n_kv_heads=1, window=37, batch=2),
+    dict(n_prefix=3100, budget=120, n_q_heads=7, n_kv_heads=1, window=32, topk_nodes=24),
 ]
 
 
