@@ -13,6 +13,9 @@
  *   - Every data pointer is a DEVICE pointer owned by the caller.  The library allocates and
  *     frees nothing; scratch comes from a caller-supplied workspace of at least
  *     graphkv_workspace_bytes(params) bytes, 256-byte aligned.
+ *     V, K_out, V_out and idx_out may instead be page-locked host memory that the device can
+ *     address (unified addressing: the same pointer): V is read only row by row for the B+W
+ *     tokens that are kept, so a cache that lives in host memory needs only Qw and K copied.
  *   - Calls validate their arguments on the host, enqueue kernels on `stream` (a cudaStream_t
  *     passed as void*; NULL = the legacy default stream) and return without synchronising.
  *     The return value reports host-side validation and launch errors only.

@@ -236,6 +236,27 @@ def test_strided_inputs(gk):
     assert torch.equal(s.cpu(), dense["scores"])
 
 
+def test_values_and_outputs_in_pinned_host_memory(gk):
+    # V is only gathered from: it may stay in page-locked host memory (same pointer on the device
+    # under unified addressing), and the compact cache may be written there directly
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=5200, budget=300, n_q_heads=8, n_kv_heads=2, batch=2)
+    inp = wl.make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    kw = cfg_kwargs(cfg)
+    ref = run_fused(gk, inp["Qw"], inp["K"], inp["V"], **kw)
+    Qd, Kd = inp["Qw"].to(dev), inp["K"].to(dev)
+    Vh = inp["V"].pin_memory()
+    p = gk.make_params(Kd, Qw=Qd, V=Vh, **kw)
+    ws = gk.alloc_workspace(p, dev)
+    K_out, _, idx, _ = gk.alloc_outputs(p, Kd, want_scores=False)
+    V_out = torch.empty(K_out.shape, dtype=K_out.dtype).pin_memory()
+    gk.graphkv_compress(p, Qd, Kd, Vh, K_out, V_out, idx, None, ws)
+    assert gk.graphkv_read_status(ws) == gk.OK          # synchronises the stream
+    assert torch.equal(idx.cpu(), ref["idx"])
+    assert torch.equal(K_out.cpu().view(torch.int16), ref["K_out"].view(torch.int16))
+    assert torch.equal(V_out.view(torch.int16), ref["V_out"].view(torch.int16))
+
+
 def test_runs_are_bitwise_repeatable(gk):
     cfg = wl.scaled(wl.LLAMA_32K, n_prefix=6000, budget=256, n_q_heads=8, n_kv_heads=2)
     inp = wl.make_inputs(cfg)
