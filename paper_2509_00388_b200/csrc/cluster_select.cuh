@@ -396,13 +396,14 @@ struct PoolSelectArgs {
 // count); each CTA lists its own, the first CTA pulls the lists through distributed shared memory
 // and ranks them by counting.  Returns false (in every CTA alike, nothing written) when they exceed kThreads; the
 // caller then runs the radix search.  `mass_hist`: kBins counts of the top 11 bits.
+// c0, c1: the histogram's counts of digits kBins-1-2t and kBins-2-2t for thread t (the caller loads
+// them early, ahead of the pooling).
 __device__ bool cluster_topk_bounded(cg::cluster_group &cl, int C, int rank, const Smem &s,
                                      const float *vals, int n_local, int base, int k,
-                                     const uint32_t *mass_hist, int *out)
+                                     uint32_t c0, uint32_t c1, int *out)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // digit b: walk the histogram from the top (thread t owns digits kBins-1-2t and kBins-2-2t)
-    const uint32_t c0 = __ldcg(mass_hist + kBins - 1 - 2 * tid), c1 = __ldcg(mass_hist + kBins - 2 - 2 * tid);
     uint32_t incl = warp_incl_scan(c0 + c1, lane);
     if (lane == 31) s.wcnt[warp] = incl;
     if (tid == 0) {
@@ -442,10 +443,13 @@ __device__ bool cluster_topk_bounded(cg::cluster_group &cl, int C, int rank, con
     __syncthreads();
     if (C > 1) cl.sync();
     // candidate t of the concatenated lists; every CTA learns the total, the first CTA pulls them
+    // (lane p reads CTA p's count, so the remote reads overlap; the walk runs on the copies)
+    uint32_t n_lane = 0;
+    if (lane < C) n_lane = C > 1 ? cl.map_shared_rank(s.misc, lane)[7] : s.misc[7];
     uint32_t total = 0;
     int mine_p = -1, mine_j = 0;
     for (int p = 0; p < C; ++p) {
-        const uint32_t n_p = C > 1 ? cl.map_shared_rank(s.misc, p)[7] : s.misc[7];
+        const uint32_t n_p = __shfl_sync(0xffffffffu, n_lane, p);
         if (n_p > (uint32_t)kThreads) total = 0x40000000u;       // a list overflowed
         if (tid >= (int)total && tid < (int)(total + n_p)) {
             mine_p = p;
@@ -474,12 +478,33 @@ __device__ bool cluster_topk_bounded(cg::cluster_group &cl, int C, int rank, con
         int *kept = s.st_idx;                              // [k] positions of the kept, unordered
         if (tid == 0) s.misc[3] = 0u;      // (word 7 may still be read by the other CTAs)
         __syncthreads();
-        for (int t = warp; t < (int)total; t += kWarps) {
-            const uint32_t kt = ck[t], pt = ci[t];
+        if (total <= (uint32_t)(kThreads / 4)) {
+            // few candidates: four threads each, every one walking a quarter of the list
+            const int t = tid >> 2, sub = tid & 3;
+            const bool live = t < (int)total;
+            const uint32_t kt = live ? ck[t] : 0u, pt = live ? ci[t] : 0u;
             int r = 0;
-            for (int u = lane; u < (int)total; u += 32) r += (ck[u] > kt) || (ck[u] == kt && ci[u] < pt);
-            r = __reduce_add_sync(0xffffffffu, r);
-            if (lane == 0 && r < k) kept[atomicAdd(&s.misc[3], 1u)] = (int)pt;
+            if (live) {
+#pragma unroll 4
+                for (int u = sub; u < (int)total; u += 4) {
+                    const uint32_t ku = ck[u], pu = ci[u];
+                    r += (int)(ku > kt) | ((int)(ku == kt) & (int)(pu < pt));
+                }
+            }
+            r += __shfl_xor_sync(0xffffffffu, r, 1);
+            r += __shfl_xor_sync(0xffffffffu, r, 2);
+            if (live && sub == 0 && r < k) kept[atomicAdd(&s.misc[3], 1u)] = (int)pt;
+        } else {
+            for (int t = warp; t < (int)total; t += kWarps) {
+                const uint32_t kt = ck[t], pt = ci[t];
+                int r = 0;
+                for (int u = lane; u < (int)total; u += 32) {
+                    const uint32_t ku = ck[u], pu = ci[u];
+                    r += (int)(ku > kt) | ((int)(ku == kt) & (int)(pu < pt));
+                }
+                r = __reduce_add_sync(0xffffffffu, r);
+                if (lane == 0 && r < k) kept[atomicAdd(&s.misc[3], 1u)] = (int)pt;
+            }
         }
         __syncthreads();
         // ascending positions: thread t places kept[t] by counting the smaller ones
@@ -511,6 +536,14 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
     if (a.zero)
         for (int i = rank * kThreads + tid; i < a.zero_words; i += C * kThreads)
             a.zero[(long long)unit * a.zero_words + i] = 0u;
+    // this thread's two counts of the mass histogram, on their way while the row is pooled
+    const bool bounded = a.mass_hist && a.k > 0 && a.k <= kThreads;
+    uint32_t hc0 = 0, hc1 = 0;
+    if (bounded) {
+        const uint32_t *mh = a.mass_hist + (long long)unit * kBins;
+        hc0 = __ldcg(mh + kBins - 1 - 2 * tid);
+        hc1 = __ldcg(mh + kBins - 2 - 2 * tid);
+    }
     if (a.a) {
         const float *row_a = a.a + (long long)unit * N;
         const int half = a.halo;
@@ -541,9 +574,7 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
     __syncthreads();
     if (a.k > 0) {
         int *out = a.src_out + (long long)unit * a.k;
-        const bool done = a.mass_hist && a.k <= kThreads &&
-                          cluster_topk_bounded(cl, C, rank, s, vals, n_local, base, a.k,
-                                               a.mass_hist + (long long)unit * kBins, out);
+        const bool done = bounded && cluster_topk_bounded(cl, C, rank, s, vals, n_local, base, a.k, hc0, hc1, out);
         if (!done) {
             const Threshold th = cluster_kth(cl, C, rank, s, vals, n_local, (uint32_t)a.k);
             cluster_emit_sorted(cl, C, rank, s, vals, n_local, base, th, out);
