@@ -90,8 +90,8 @@ def algorithmic_bytes(cfg, kernel: str) -> float:
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
 # summarised in profiles/kernels_llama31_8b_32k_ncu_full.md; cold cache.  Only for the workload
 # and kernels that capture covers; anything else reports null.
-NCU_TRAFFIC = {"llama31_8b_32k": {"score_stats_tc": 68.14e6, "score_emit_tc": 67.91e6,
-                                  "pool_select_sources": 1.18e6, "similarity_tc": 67.73e6,
+NCU_TRAFFIC = {"llama31_8b_32k": {"score_stats_tc": 67.86e6, "score_emit_tc": 67.87e6,
+                                  "pool_select_sources": 1.18e6, "similarity_tc": 67.66e6,
                                   "decay_select_gather": 4.66e6}}
 
 
