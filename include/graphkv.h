@@ -160,6 +160,20 @@ graphkv_status graphkv_read_status(const void *workspace, void *stream);
 
 const char *graphkv_status_string(graphkv_status status);
 
+/* ---- diagnostics (the paper has no counterpart: inspection support of this library) -----------
+ * graphkv_read_neighbors: copies the neighbourhoods N(o_i) of Eq. 3 that the last graphkv_propagate
+ * or graphkv_compress on this workspace built, as they were applied by the decay rounds:
+ *   nbr_idx_out [batch][n_kv_heads][k][m] int32  positions of each source's m neighbours
+ *   nbr_e_out   [batch][n_kv_heads][k][m] fp32   their cosines e_ij
+ * (device pointers; either may be NULL), row i of a head belonging to the i-th source in the
+ * order graphkv_propagate reports the sources (ascending position); the order within a row
+ * carries no meaning.  m = graphkv_resolve_neighbors(N, params.neighbors).
+ * The copies are enqueued on `stream` after that call; `params` must be the ones it was given.
+ * Returns GRAPHKV_ERR_INVALID_ARG when those params build no graph (topk_nodes, rounds or m zero). */
+graphkv_status graphkv_read_neighbors(const graphkv_params *params, const void *workspace,
+                                      size_t workspace_bytes, int32_t *nbr_idx_out,
+                                      float *nbr_e_out, void *stream);
+
 /* ---- tracing (the paper has no counterpart: measurement support of this library) -------------
  * graphkv_launch_count: kernels this process has launched through the library so far.
  * graphkv_trace_enable(1): from now on every kernel launch is bracketed by a pair of CUDA events

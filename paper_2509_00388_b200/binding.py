@@ -24,7 +24,7 @@ EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_scor
            "graphkv_propagate", "graphkv_select_gather", "graphkv_compress",
            "graphkv_read_status", "graphkv_status_string", "graphkv_launch_count",
            "graphkv_trace_enable", "graphkv_trace_read", "graphkv_builtin_scratch_needed",
-           "graphkv_score_noalloc", "graphkv_read_status_noalloc")
+           "graphkv_score_noalloc", "graphkv_read_status_noalloc", "graphkv_read_neighbors")
 
 
 class GraphKVError(RuntimeError):
@@ -75,6 +75,8 @@ def lib() -> C.CDLL:
         L.graphkv_compress.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.graphkv_read_status.restype = C.c_int
         L.graphkv_read_status.argtypes = [vp, vp]
+        L.graphkv_read_neighbors.restype = C.c_int
+        L.graphkv_read_neighbors.argtypes = [P, vp, sz, vp, vp, vp]
         L.graphkv_builtin_scratch_needed.restype = sz
         L.graphkv_builtin_scratch_needed.argtypes = [P]
         L.graphkv_score_noalloc.restype = C.c_int
@@ -206,6 +208,13 @@ def graphkv_compress(p: Params, Qw: torch.Tensor, K: torch.Tensor, V: torch.Tens
 
 def graphkv_read_status(ws: torch.Tensor) -> int:
     return int(lib().graphkv_read_status(_ptr(ws), _stream(ws.device)))
+
+
+def graphkv_read_neighbors(p: Params, ws: torch.Tensor, nbr_idx_out: Optional[torch.Tensor],
+                           nbr_e_out: Optional[torch.Tensor]) -> None:
+    _check(lib().graphkv_read_neighbors(C.byref(p), _ptr(ws), ws.numel(), _ptr(nbr_idx_out),
+                                        _ptr(nbr_e_out), _stream(ws.device)),
+           "graphkv_read_neighbors")
 
 
 def graphkv_launch_count() -> int:

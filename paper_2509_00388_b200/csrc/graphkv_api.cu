@@ -805,6 +805,28 @@ graphkv_status graphkv_read_status(const void *workspace, void *stream)
     return static_cast<graphkv_status>(word);
 }
 
+graphkv_status graphkv_read_neighbors(const graphkv_params *params, const void *workspace,
+                                      size_t workspace_bytes, int32_t *nbr_idx_out,
+                                      float *nbr_e_out, void *stream)
+{
+    Dims d;
+    graphkv_status rc = resolve(params, &d);
+    if (rc != GRAPHKV_OK) return rc;
+    if (!graph_active(d)) return GRAPHKV_ERR_INVALID_ARG;
+    const Layout l = layout_of(d);
+    if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t pairs = (size_t)d.units * d.K_src * d.m;
+    const unsigned char *ws = static_cast<const unsigned char *>(workspace);
+    if (nbr_idx_out && cudaMemcpyAsync(nbr_idx_out, ws + l.nbr_idx, pairs * sizeof(int),
+                                       cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return GRAPHKV_ERR_CUDA;
+    if (nbr_e_out && cudaMemcpyAsync(nbr_e_out, ws + l.nbr_e, pairs * sizeof(float),
+                                     cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return GRAPHKV_ERR_CUDA;
+    return GRAPHKV_OK;
+}
+
 int64_t graphkv_launch_count(void) { return g_launches.load(); }
 
 void graphkv_trace_enable(int32_t enable)

@@ -7,11 +7,11 @@
 // 128 x NP dot products against the source keys into its own TMEM columns, and the epilogue
 // threads (thread = key) take the key's norm from the staged tile.  When the sweep is over the
 // chunk's whole edge block still sits in TMEM, and the CTA
-//   1. takes, per source, a threshold tau that at least m eligible edges of the chunk reach:
-//      the lower edge of the highest cosine bin such that m+1 of the per-thread maxima lie in or
-//      above it (distinct threads hold distinct keys, and at most one of them is the source
-//      itself);
-//   2. re-reads TMEM and lists the edges >= tau, excluding the source itself;
+//   1. takes, per source, a threshold bin that at least m eligible edges of the chunk reach:
+//      the highest cosine bin such that m+1 of the per-thread maxima lie in or above it (distinct
+//      threads hold distinct keys, and at most one of them is the source itself);
+//   2. re-reads TMEM and lists the edges whose bin (the same expression as in step 1, so that a
+//      counted maximum is always listed) reaches it, excluding the source itself;
 //   3. if a list outgrows its capacity (many ties), finds that source's exact m-th largest
 //      (edge descending, position ascending) by bisection over counting passes and lists
 //      exactly those m.
@@ -54,7 +54,7 @@ template <int NP> __host__ __device__ constexpr int sim_tiles_cap() { return 512
 template <int NP> __host__ __device__ inline size_t sim_smem_bytes(int stages)
 {
     return 1024 + (size_t)NP * 256 + (size_t)stages * kTileBytes + (8 + 8 + kSimMaxTiles) * 8 + 16 +
-           (size_t)sim_tiles_cap<NP>() * 128 * 4 + (size_t)NP * 4 * 4 + (size_t)NP * kCandCap * 8 + 64;
+           (size_t)sim_tiles_cap<NP>() * 128 * 4 + (size_t)NP * 5 * 4 + (size_t)NP * kCandCap * 8 + 64;
 }
 
 template <int NP>
@@ -90,12 +90,13 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     const uint32_t s_tmem = s_done0 + kSimMaxTiles * 8;
     const uint32_t s_invn = s_tmem + 16;
     const uint32_t s_book = s_invn + kTilesCap * 128 * 4;
-    const uint32_t s_list = s_book + NP * 4 * 4;
+    const uint32_t s_list = s_book + NP * 5 * 4;
     float *inv_norm = reinterpret_cast<float *>(gen + (s_invn - base));        // [tile][128]
     int *src_pos = reinterpret_cast<int *>(gen + (s_book - base));              // [NP]
     float *src_inv = reinterpret_cast<float *>(src_pos + NP);                   // [NP]
     float *tau = src_inv + NP;                                                  // [NP] threshold cosine
     int *cnt = reinterpret_cast<int *>(tau + NP);                               // [NP]
+    int *tau_bin = cnt + NP;                                                    // [NP] bin whose lower edge tau is
     Cand *list = reinterpret_cast<Cand *>(gen + (s_list - base));               // [NP][kCandCap]
     // after the sweep the stage memory holds the bins of the maxima and the threads' edge queues
     // (a key position takes 26 bits there: rows this kernel is given are shorter than 2^18 keys)
@@ -312,20 +313,22 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 if (lane < 4 && g * 4 + lane < d.K_src) {
                     const uint32_t bs = lane == 0 ? bstar[0] : lane == 1 ? bstar[1] : lane == 2 ? bstar[2] : bstar[3];
                     tau[g * 4 + lane] = bs == 0 ? -1.0f : (float)bs * (2.0f / kMaxBins) - 1.0f;
+                    tau_bin[g * 4 + lane] = (int)bs;
                 }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            // 2. list the edges that reach the threshold.  theta is the threshold brought to the scale
-            //    of dot / |k_j|, lowered by a few ulps so that no edge with cosine >= tau is missed.
+            // 2. list the edges that reach the threshold bin.  theta is the bin's lower edge brought to
+            //    the scale of dot / |k_j|, lowered (the bin index rounds: a cosine a few 1e-8 under
+            //    the edge still lands in the bin) so that no edge of the bin is missed.
             //    Straight-line code: a thread appends the few edges of its keys that pass, as
             //    (value, source and key), to a queue of its own; afterwards it turns each into a
-            //    cosine, checks it against tau itself and adds it to the source's list (the order
+            //    cosine, checks its bin against the threshold bin and adds it to the source's list (the order
             //    within a list carries no meaning).  A queue that fills up sends every source of the
             //    chunk down the exact path of step 3.
             float theta[NP];
 #pragma unroll
             for (int c = 0; c < NP; ++c) {
-                const float q = c < d.K_src ? tau[c] / src_inv[c] : INFINITY;
+                const float q = c < d.K_src ? (tau[c] - 2.4e-7f) / src_inv[c] : INFINITY;
                 theta[c] = q - fabsf(q) * 2.4e-7f - 1e-30f;
             }
             // (branch-free, the store and the count under one predicate; a key past the end of the
@@ -359,7 +362,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 const uint2 en = q0[k * kSimEpiThreads];
                 const int c = en.y >> 26, j = en.y & 0x3ffffffu;
                 const float e = fminf(fmaxf(__uint_as_float(en.x) * src_inv[c], -1.0f), 1.0f);
-                if (e >= tau[c] && j != src_pos[c]) {
+                const int bin = min(max(static_cast<int>((e + 1.0f) * (kMaxBins / 2)), 0), kMaxBins - 1);
+                if (bin >= tau_bin[c] && j != src_pos[c]) {
                     const int pos = atomicAdd(&cnt[c], 1);
                     if (pos < kCandCap) list[c * kCandCap + pos] = Cand{e, j};
                 }

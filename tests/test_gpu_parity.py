@@ -36,6 +36,12 @@ def run_staged(gk, Qw, K, V, **kw):
     gk.graphkv_propagate(p, Kd, s, src, ws)
     if src is not None:
         out["src"] = src.cpu()
+    m = gk.resolve_neighbors(p.seq_len - p.window, p.neighbors)
+    if src is not None and p.rounds > 0 and m > 0:
+        nbr = torch.empty((p.batch, p.n_kv_heads, p.topk_nodes, m), dtype=torch.int32, device=dev)
+        nbr_e = torch.empty(nbr.shape, dtype=torch.float32, device=dev)
+        gk.graphkv_read_neighbors(p, ws, nbr, nbr_e)
+        out.update(nbr=nbr.cpu(), nbr_e=nbr_e.cpu())
     out["scores"] = s.cpu()
     gk.graphkv_select_gather(p, s, Kd, Vd, K_out, V_out, idx, ws)
     assert gk.graphkv_read_status(ws) == gk.OK
@@ -51,7 +57,13 @@ def run_fused(gk, Qw, K, V, **kw):
     K_out, V_out, idx, s = gk.alloc_outputs(p, Kd)
     gk.graphkv_compress(p, Qd, Kd, Vd, K_out, V_out, idx, s, ws)
     assert gk.graphkv_read_status(ws) == gk.OK
-    return {"idx": idx.cpu(), "K_out": K_out.cpu(), "V_out": V_out.cpu(), "scores": s.cpu()}
+    out = {"idx": idx.cpu(), "K_out": K_out.cpu(), "V_out": V_out.cpu(), "scores": s.cpu()}
+    m = gk.resolve_neighbors(p.seq_len - p.window, p.neighbors)
+    if p.topk_nodes > 0 and p.rounds > 0 and m > 0:
+        nbr = torch.empty((p.batch, p.n_kv_heads, p.topk_nodes, m), dtype=torch.int32, device=dev)
+        gk.graphkv_read_neighbors(p, ws, nbr, None)
+        out["nbr"] = nbr.cpu()
+    return out
 
 
 def cfg_kwargs(cfg, layer=0):
@@ -69,9 +81,17 @@ def check(gk, cfg, layer=0, sequences=None, strict_overlap=True, **override):
     for name in ("idx", "K_out", "V_out", "scores"):
         assert torch.equal(staged[name].view(torch.uint8), fused[name].view(torch.uint8)), \
             f"fused compress differs from the staged calls in {name}"
+    if "nbr" in fused:
+        assert torch.equal(torch.sort(staged["nbr"], dim=-1).values,
+                           torch.sort(fused["nbr"], dim=-1).values), \
+            "fused compress built other neighbourhoods than the staged calls"
     rep = pu.check_compress(staged, inp["Qw"], inp["K"], inp["V"], strict_overlap=strict_overlap,
                             **kw)
     print(json.dumps({"config": cfg.name, "layer": layer, **rep.as_dict()}))
+    if cfg == wl.CONFIGS.get(cfg.name) and not override:
+        tag = cfg.name + (f"_layer{layer}" if cfg.n_layers > 1 else "") + \
+            ("" if sequences is None else "_seq" + "".join(str(q) for q in sequences))
+        rep.write(tag)
     return rep
 
 
@@ -263,7 +283,7 @@ def test_runs_are_bitwise_repeatable(gk):
     a = run_fused(gk, inp["Qw"], inp["K"], inp["V"], **cfg_kwargs(cfg))
     b = run_fused(gk, inp["Qw"], inp["K"], inp["V"], **cfg_kwargs(cfg))
     for name in a:
-        assert torch.equal(a[name].view(torch.uint8), b[name].view(torch.uint8))
+        assert torch.equal(a[name].view(torch.uint8), b[name].view(torch.uint8)), name
 
 
 def test_select_gather_alone_is_bit_exact_with_planted_ties(gk):

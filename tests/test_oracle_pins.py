@@ -324,6 +324,10 @@ def test_adaptive_neighbour_rule():
     assert okv.resolve_neighbors(32768, 0) == 32
     assert okv.resolve_neighbors(131072, 0) == 32
     assert okv.resolve_neighbors(32768, 5) == 5
+    # the length rule is a factor of 1e-3 (not 2^-10), floored
+    assert okv.resolve_neighbors(5000, 0) == 5
+    assert okv.resolve_neighbors(31999, 0) == 31
+    assert okv.resolve_neighbors(1999, 0) == 1 and okv.resolve_neighbors(2000, 0) == 2
 
 
 # ----------------------------------------------------------------------------- step (IV)
