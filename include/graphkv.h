@@ -189,6 +189,16 @@ int64_t graphkv_launch_count(void);
 void graphkv_trace_enable(int32_t enable);
 int32_t graphkv_trace_read(graphkv_trace_record *out, int32_t capacity);
 
+/* graphkv_phase_timing_read: only a library built with -DGRAPHKV_PHASE_TIMING keeps, per kernel, the
+ * time its CTAs spent between the phase marks in its source (one thread per CTA reads the global
+ * timer).  Synchronises the device, copies out and clears the tables:
+ *   out[(k * 24 + i) * 2]     nanoseconds summed over CTAs, kernel k, phase i (i = 0: whole CTA)
+ *   out[(k * 24 + i) * 2 + 1] the largest single value
+ *   out[8 * 24 * 2 + k]       CTAs counted for kernel k
+ * `out` is a HOST array of 8 * 24 * 2 + 8 words.  Returns 1, or 0 (nothing written) when the
+ * library was built without the option. */
+int32_t graphkv_phase_timing_read(uint64_t *out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,7 @@ EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_scor
            "graphkv_propagate", "graphkv_select_gather", "graphkv_compress",
            "graphkv_read_status", "graphkv_status_string", "graphkv_launch_count",
            "graphkv_trace_enable", "graphkv_trace_read", "graphkv_builtin_scratch_needed",
-           "graphkv_score_noalloc", "graphkv_read_status_noalloc", "graphkv_read_neighbors")
+           "graphkv_score_noalloc", "graphkv_read_status_noalloc", "graphkv_read_neighbors", "graphkv_phase_timing_read")
 
 
 class GraphKVError(RuntimeError):
@@ -77,6 +77,8 @@ def lib() -> C.CDLL:
         L.graphkv_read_status.argtypes = [vp, vp]
         L.graphkv_read_neighbors.restype = C.c_int
         L.graphkv_read_neighbors.argtypes = [P, vp, sz, vp, vp, vp]
+        L.graphkv_phase_timing_read.restype = C.c_int32
+        L.graphkv_phase_timing_read.argtypes = [C.POINTER(C.c_uint64)]
         L.graphkv_builtin_scratch_needed.restype = sz
         L.graphkv_builtin_scratch_needed.argtypes = [P]
         L.graphkv_score_noalloc.restype = C.c_int
@@ -230,6 +232,22 @@ def graphkv_trace_read(capacity: int = 1 << 16):
     buf = (TraceRecord * capacity)()
     n = lib().graphkv_trace_read(buf, capacity)
     return [(buf[i].name.decode(), float(buf[i].ms)) for i in range(n)]
+
+
+def graphkv_phase_timing_read():
+    """Per-kernel phase times of a library built with GRAPHKV_PHASE_TIMING, or None.
+    Returns {kernel index: (CTAs, [(mean ns, max ns) per phase])}; phase 0 is the whole CTA."""
+    n_k, n_s = 8, 24
+    buf = (C.c_uint64 * (n_k * n_s * 2 + n_k))()
+    if not lib().graphkv_phase_timing_read(buf):
+        return None
+    out = {}
+    for k in range(n_k):
+        cnt = buf[n_k * n_s * 2 + k]
+        if cnt:
+            out[k] = (int(cnt), [(buf[(k * n_s + i) * 2] / cnt, int(buf[(k * n_s + i) * 2 + 1]))
+                                 for i in range(n_s)])
+    return out
 
 
 def alloc_outputs(p: Params, like: torch.Tensor, want_scores: bool = True

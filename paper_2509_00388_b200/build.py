@@ -33,20 +33,25 @@ def _stale() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
+def build(force: bool = False, verbose: bool = False, phase_timing: bool = False) -> str:
+    """The library; with phase_timing, a second one (libgraphkv_phases.so) whose kernels stamp the
+    global timer at their phase marks (point GRAPHKV_LIB at it)."""
+    lib = LIB.replace(".so", "_phases.so") if phase_timing else LIB
+    if not force and not phase_timing and not _stale():
+        return lib
+    tmp = lib + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17",
            "-lineinfo", "-Xcompiler", "-fPIC",
            "-shared", "-I", INCLUDE, "-I", CSRC, "-o", tmp] + sources()
+    if phase_timing:
+        cmd.insert(1, "-DGRAPHKV_PHASE_TIMING")
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, phase_timing="--phases" in sys.argv))

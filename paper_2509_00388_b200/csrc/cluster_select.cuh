@@ -33,22 +33,29 @@ constexpr int kMaxPerThread = kMaxChunk / kThreads;
 constexpr int kStage = 2048;           // neighbour-list entries staged in shared memory at a time
 constexpr int kMergeWarps = 8;         // groups of four warps of a CTA, one source each at a time
 constexpr int kSurvCap = 256;          // merged candidates one warp ranks in shared memory
+constexpr int kFineBins = 8192;        // one-pass selection: histogram over the top 13 bits of the ordered image
+constexpr int kFineShift = 19;
+constexpr int kTotWords = kFineBins / 2;   // a CTA's slice of the cluster-wide fine histogram (C >= 2)
 static_assert(kMergeWarps * kSurvCap * sizeof(Cand) <= 2 * kStage * 4, "survivors reuse the staging area");
 
 // Shared-memory carve-up common to both kernels (dynamic shared memory, 16-byte aligned).
 struct Smem {
     uint32_t *hist;       // [kBins] this CTA's digit histogram
-    uint32_t *tot;        // [kBins] cluster-wide histogram (every CTA holds a copy)
+    uint32_t *tot;        // [kTotWords] cluster-wide histogram (every CTA holds a copy / its slice)
+    uint32_t *fine;       // [kFineBins] this CTA's fine histogram
     uint32_t *wcnt;       // [2 * kWarps] per-warp counts
-    uint32_t *misc;       // [16] broadcast words and this CTA's published counts
-    int *st_idx;          // [kStage] staged neighbour positions, relative to the chunk
-    float *st_f;          // [kStage] their decay factors
+    uint32_t *misc;       // [32] broadcast words and this CTA's published counts
+    int *st_idx;          // [kStage] staging: neighbour positions / candidate positions / survivors
+    float *st_f;          // [kStage] staging: decay factors / survivors
+    int *nb_j;            // [kStage] the unit's neighbour lists, positions (every CTA holds a copy)
+    float *nb_f;          // [kStage] their decay factors over all rounds
     float *vals;          // [halo + chunk + halo]
 };
 
 __host__ __device__ inline size_t smem_bytes(int chunk, int halo)
 {
-    return (size_t)(2 * kBins + 2 * kWarps + 16 + 2 * kStage) * 4 + (size_t)(chunk + 2 * halo + 8) * 4;
+    return (size_t)(kBins + kTotWords + kFineBins + 2 * kWarps + 32 + 4 * kStage) * 4 +
+           (size_t)(chunk + 2 * halo + 8) * 4;
 }
 
 __device__ __forceinline__ Smem carve(uint8_t *raw, int halo)
@@ -56,11 +63,14 @@ __device__ __forceinline__ Smem carve(uint8_t *raw, int halo)
     Smem s;
     s.hist = reinterpret_cast<uint32_t *>(raw);
     s.tot = s.hist + kBins;
-    s.wcnt = s.tot + kBins;
+    s.fine = s.tot + kTotWords;
+    s.wcnt = s.fine + kFineBins;
     s.misc = s.wcnt + 2 * kWarps;
-    s.st_idx = reinterpret_cast<int *>(s.misc + 16);
+    s.st_idx = reinterpret_cast<int *>(s.misc + 32);
     s.st_f = reinterpret_cast<float *>(s.st_idx + kStage);
-    s.vals = s.st_f + kStage;
+    s.nb_j = reinterpret_cast<int *>(s.st_f + kStage);
+    s.nb_f = reinterpret_cast<float *>(s.nb_j + kStage);
+    s.vals = s.nb_f + kStage;
     (void)halo;
     return s;
 }
@@ -69,6 +79,16 @@ __device__ __forceinline__ Smem carve(uint8_t *raw, int halo)
 // whose masked key equals it the `remaining` lowest indices.
 struct Threshold {
     uint32_t prefix, mask, remaining;
+};
+
+// The elements a selection ranks: all n of a chunk in shared memory (list == nullptr), or the n
+// of them whose chunk-relative positions `list` holds in ascending order.
+struct RowView {
+    const float *vals;
+    const int *list;
+    int n;
+    __device__ __forceinline__ int pos(int t) const { return list ? list[t] : t; }
+    __device__ __forceinline__ float at(int t) const { return vals[pos(t)]; }
 };
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane)
@@ -85,8 +105,9 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane)
 // All CTAs of the cluster call this with the same k (1 <= k <= elements in the row) and return
 // the same Threshold.  Executes the same number of cluster barriers in every CTA.
 __device__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const Smem &s,
-                                 const float *vals, int n_local, uint32_t k)
+                                 const RowView &row, uint32_t k)
 {
+    const int n_local = row.n;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     Threshold th{0u, 0u, k};
 #pragma unroll 1
@@ -100,7 +121,7 @@ __device__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const S
             bool valid = i < n_local;
             uint32_t bin = 0;
             if (valid) {
-                const uint32_t u = float_to_key(vals[i]);
+                const uint32_t u = float_to_key(row.at(i));
                 valid = (u & th.mask) == th.prefix;
                 bin = (u >> shift) & (nb - 1u);
             }
@@ -163,14 +184,296 @@ __device__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const S
     return th;
 }
 
+// Candidates for the k largest of a chunk in shared memory.  The chunk's elements fall into
+// groups (a thread's strided elements, cut into runs); the k-th largest of the groups' maxima
+// bounds the k-th largest element from below, because distinct groups hold distinct elements.
+// The bound is taken as the lower edge of the fine-histogram bin of that maximum; the elements
+// that reach it (about twice k when a group holds n / 2k elements) are listed by ascending
+// position in `list`.  Returns their number, or -1 when grouping cannot help (k above a quarter
+// of the chunk) or the list would outgrow `cap`; the caller then ranks the whole chunk.
+// Any chunk's bound also holds for a longer row the chunk is part of.
+__device__ int filter_candidates(const Smem &s, const float *vals, int n_local, uint32_t k,
+                                 int *list, int cap)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = ceil_div(n_local, kThreads);                       // strided elements per thread
+    const int gpt = min(per, ceil_div(2 * (int)k, kThreads));          // groups per thread
+    const int g = gpt > 0 ? ceil_div(per, gpt) : 0;                    // elements per group
+    if (g < 2 || k > (uint32_t)n_local) return -1;
+    for (int i = tid; i < kFineBins; i += kThreads) s.fine[i] = 0u;
+    __syncthreads();
+    for (int q0 = 0; q0 < per; q0 += g) {
+        float best = -INFINITY;
+        bool any = false;
+        for (int q = q0; q < min(q0 + g, per); ++q) {
+            const int i = q * kThreads + tid;
+            if (i < n_local) {
+                best = fmaxf(best, vals[i]);
+                any = true;
+            }
+        }
+        if (any) atomicAdd(&s.fine[float_to_key(best) >> kFineShift], 1u);
+    }
+    __syncthreads();
+    // the bin of the k-th largest maximum: thread t owns bins kFineBins-1-8t-q, q < 8
+    uint32_t c[8], sum = 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        c[q] = s.fine[kFineBins - 1 - (tid * 8 + q)];
+        sum += c[q];
+    }
+    uint32_t incl = warp_incl_scan(sum, lane);
+    if (lane == 31) s.wcnt[warp] = incl;
+    if (tid == 0) s.misc[23] = 0u;              // bin 0 (everything passes) with fewer than k groups
+    __syncthreads();
+    if (warp == 0) s.wcnt[lane] = warp_incl_scan(s.wcnt[lane], lane);
+    __syncthreads();
+    incl += warp == 0 ? 0u : s.wcnt[warp - 1];
+    uint32_t run = incl - sum;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        if (run < k && run + c[q] >= k) s.misc[23] = (uint32_t)(kFineBins - 1 - (tid * 8 + q));
+        run += c[q];
+    }
+    __syncthreads();
+    const uint32_t bound = s.misc[23] << kFineShift;
+    // ordered listing: warp w owns the contiguous segment [w * seg, (w + 1) * seg)
+    const int seg = ((n_local + kWarps - 1) / kWarps + 31) & ~31;
+    const int lo = min(warp * seg, n_local), hi = min(lo + seg, n_local);
+    uint32_t cnt = 0;
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        const int i = i0 + lane;
+        cnt += __popc(__ballot_sync(0xffffffffu, i < hi && float_to_key(vals[i]) >= bound));
+    }
+    if (lane == 0) s.wcnt[kWarps + warp] = cnt;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t v = s.wcnt[kWarps + lane], vi = warp_incl_scan(v, lane);
+        s.wcnt[kWarps + lane] = vi - v;
+        if (lane == 31) s.misc[23] = vi;
+    }
+    __syncthreads();
+    const int total = (int)s.misc[23];
+    if (total > cap) return -1;
+    uint32_t off = s.wcnt[kWarps + warp];
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        const int i = i0 + lane;
+        const bool keep = i < hi && float_to_key(vals[i]) >= bound;
+        const unsigned bm = __ballot_sync(0xffffffffu, keep);
+        if (keep) list[off + __popc(bm & ((1u << lane) - 1u))] = i;
+        off += __popc(bm);
+    }
+    __syncthreads();
+    return total;
+}
+
+// k-th largest of the cluster's row in one histogram pass: a kFineBins histogram over the top 13
+// bits of the ordered image (sign, exponent, four mantissa bits: sixteen bins per octave), reduced
+// across the cluster in slices; the bin b* that holds the k-th largest is located by every CTA
+// alike; the elements above it are kept, and the few inside it are pulled by the first CTA and
+// ranked by counting (value descending, position ascending), which gives the exact threshold
+// value and the number of its ties to keep.  Falls back to the three-digit search when b* holds
+// more than a few hundred elements (large budgets, rows with massive ties).  Same contract as cluster_kth.
+__device__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                      const RowView &row, int base, uint32_t k, PhaseClock &pc)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_local = row.n;
+    for (int i = tid; i < kFineBins; i += kThreads) s.fine[i] = 0u;
+    if (tid == 0) s.misc[17] = 0u;                     // this CTA's candidate counter
+    __syncthreads();
+    for (int i0 = 0; i0 < n_local; i0 += kThreads) {
+        const int i = i0 + tid;
+        const bool valid = i < n_local;
+        const uint32_t bin = valid ? float_to_key(row.at(i)) >> kFineShift : 0u;
+        // lanes sharing the first valid lane's bin are counted with one atomic (scores of a row
+        // crowd into few bins); the others add for themselves
+        const unsigned vm = __ballot_sync(0xffffffffu, valid);
+        if (vm) {
+            const int leader = __ffs(vm) - 1;
+            const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
+            const bool same = valid && bin == lbin;
+            const unsigned sm = __ballot_sync(0xffffffffu, same);
+            if (lane == leader) atomicAdd(&s.fine[lbin], (uint32_t)__popc(sm));
+            else if (valid && !same) atomicAdd(&s.fine[bin], 1u);
+        }
+    }
+    __syncthreads();
+    pc.mark();
+    // cluster-wide counts of this CTA's slice of the bins, and the slice's total
+    const int slice = kFineBins / C;
+    uint32_t mine = 0;
+    if (C > 1) {
+        cl.sync();                                       // every CTA's histogram is complete
+        for (int b = tid; b < slice; b += kThreads) {
+            uint32_t sum = 0;
+            for (int p = 0; p < C; ++p) sum += cl.map_shared_rank(s.fine, p)[rank * slice + b];
+            s.tot[b] = sum;
+            mine += sum;
+        }
+    } else {
+        for (int b = tid; b < slice; b += kThreads) mine += s.fine[b];
+    }
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    if (lane == 0) s.wcnt[warp] = mine;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t t = __reduce_add_sync(0xffffffffu, s.wcnt[lane]);
+        if (lane == 0) s.misc[16] = t;
+    }
+    __syncthreads();
+    pc.mark();
+    if (C > 1) cl.sync();                                // slices and their totals are complete
+    pc.mark();
+    // the slice that holds the k-th largest (rank C-1 has the highest bins)
+    uint32_t s_lane = 0;
+    if (lane < C) s_lane = C > 1 ? cl.map_shared_rank(s.misc, lane)[16] : s.misc[16];
+    uint32_t above = 0;
+    int rstar = 0;
+    for (int p = C - 1; p >= 0; --p) {
+        const uint32_t sp = __shfl_sync(0xffffffffu, s_lane, p);
+        if (above + sp >= k) { rstar = p; break; }
+        above += sp;
+    }
+    // walk that slice from its top bin: thread t owns bins slice-1-t*per-q, q < per
+    const uint32_t *tt = C > 1 ? cl.map_shared_rank(s.tot, rstar) : s.fine;
+    const int per = slice / kThreads;                    // 1, 2, 4 or 8
+    uint32_t c[8], sum = 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        c[q] = q < per ? tt[slice - 1 - (tid * per + q)] : 0u;
+        sum += c[q];
+    }
+    uint32_t incl = warp_incl_scan(sum, lane);
+    if (lane == 31) s.wcnt[kWarps + warp] = incl;
+    __syncthreads();
+    if (warp == 0) s.wcnt[kWarps + lane] = warp_incl_scan(s.wcnt[kWarps + lane], lane);
+    __syncthreads();
+    incl += warp == 0 ? 0u : s.wcnt[kWarps + warp - 1];
+    uint32_t run = above + incl - sum;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        if (q < per && run < k && run + c[q] >= k) {
+            s.misc[20] = (uint32_t)(rstar * slice + slice - 1 - (tid * per + q));
+            s.misc[21] = run;
+            s.misc[22] = c[q];
+        }
+        run += c[q];
+    }
+    __syncthreads();
+    pc.mark();
+    const uint32_t bstar = s.misc[20], n_above = s.misc[21], n_in = s.misc[22];
+    const uint32_t need = k - n_above;                   // of the n_in elements in bin b*
+    if (need == n_in) return Threshold{bstar << kFineShift, (uint32_t)(kFineBins - 1) << kFineShift, n_in};
+    if (n_in > (uint32_t)kThreads / 4) return cluster_kth(cl, C, rank, s, row, k);     // too many to rank by counting
+    // this CTA's elements of bin b* -> its own lists (keys and positions in the two halves of hist):
+    // every warp counts its own first, a scan over the warps gives each its slots
+    uint32_t *ck = s.hist;
+    int *ci = reinterpret_cast<int *>(s.hist + kThreads);
+    uint32_t mine_n = 0;
+    for (int i0 = 0; i0 < n_local; i0 += kThreads) {
+        const int i = i0 + tid;
+        const bool cand = i < n_local && (float_to_key(row.at(i)) >> kFineShift) == bstar;
+        mine_n += __popc(__ballot_sync(0xffffffffu, cand));
+    }
+    if (lane == 0) s.wcnt[warp] = mine_n;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t v = s.wcnt[lane], vi = warp_incl_scan(v, lane);
+        s.wcnt[lane] = vi - v;
+        if (lane == 31) s.misc[17] = vi;
+    }
+    __syncthreads();
+    uint32_t slot0 = s.wcnt[warp];
+    for (int i0 = 0; i0 < n_local; i0 += kThreads) {
+        const int i = i0 + tid;
+        uint32_t key = 0;
+        bool cand = false;
+        int at = 0;
+        if (i < n_local) {
+            at = row.pos(i);
+            key = float_to_key(row.vals[at]);
+            cand = (key >> kFineShift) == bstar;
+        }
+        const unsigned bm = __ballot_sync(0xffffffffu, cand);
+        if (cand) {
+            const uint32_t slot = slot0 + __popc(bm & ((1u << lane) - 1u));
+            ck[slot] = key;
+            ci[slot] = base + at;
+        }
+        slot0 += __popc(bm);
+    }
+    __syncthreads();
+    pc.mark();
+    if (C > 1) cl.sync();                                // every CTA's list is complete
+    pc.mark();
+    if (rank == 0) {
+        uint32_t n_lane = 0;
+        if (lane < C) n_lane = C > 1 ? cl.map_shared_rank(s.misc, lane)[17] : s.misc[17];
+        uint32_t total = 0;
+        int mine_p = -1, mine_j = 0;
+        for (int p = 0; p < C; ++p) {
+            const uint32_t n_p = __shfl_sync(0xffffffffu, n_lane, p);
+            if (tid >= (int)total && tid < (int)(total + n_p)) {
+                mine_p = p;
+                mine_j = tid - (int)total;
+            }
+            total += n_p;
+        }
+        uint32_t key = 0;
+        int pos = 0;
+        if (mine_p >= 0) {
+            key = (C > 1 ? cl.map_shared_rank(ck, mine_p) : ck)[mine_j];
+            pos = (C > 1 ? cl.map_shared_rank(ci, mine_p) : ci)[mine_j];
+        }
+        __syncthreads();                                 // own list read before it is overwritten
+        if (mine_p >= 0) {
+            ck[tid] = key;
+            ci[tid] = pos;
+        }
+        __syncthreads();
+        {
+            // few candidates (at most kThreads / 4): four threads each, every one walking a quarter of the list
+            const int t = tid >> 2, sub = tid & 3;
+            const bool live = t < (int)total;
+            const uint32_t kt = live ? ck[t] : 0u;
+            const int pt = live ? ci[t] : 0;
+            uint32_t r = 0, n_gt = 0;                    // rank among all; candidates with a larger value
+            if (live) {
+#pragma unroll 4
+                for (int u = sub; u < (int)total; u += 4) {
+                    const uint32_t ku = ck[u];
+                    const int pu = ci[u];
+                    n_gt += ku > kt;
+                    r += (ku > kt) | ((ku == kt) & (pu < pt));
+                }
+            }
+            r += __shfl_xor_sync(0xffffffffu, r, 1);
+            r += __shfl_xor_sync(0xffffffffu, r, 2);
+            n_gt += __shfl_xor_sync(0xffffffffu, n_gt, 1);
+            n_gt += __shfl_xor_sync(0xffffffffu, n_gt, 2);
+            if (live && sub == 0 && r == need - 1) {
+                s.misc[18] = kt;
+                s.misc[19] = need - n_gt;
+            }
+        }
+        __syncthreads();
+    }
+    pc.mark();
+    if (C > 1) cl.sync();                                // the first CTA's answer is published
+    pc.mark();
+    const uint32_t *m0 = C > 1 ? cl.map_shared_rank(s.misc, 0) : s.misc;
+    return Threshold{m0[18], 0xffffffffu, m0[19]};
+}
+
 // Ascending positions of the kept elements of the cluster's row -> out[0..k).  Returns nothing;
 // ends with the writes of this CTA issued (callers fence before another CTA reads them).
 // One cluster barrier.
 __device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, const Smem &s,
-                                    const float *vals, int n_local, int base, Threshold th,
-                                    int *out)
+                                    const RowView &row, int base, Threshold th, int *out)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_local = row.n;
     // warp w owns the contiguous segment [w * seg, (w + 1) * seg) of the chunk
     const int seg = ((n_local + kWarps - 1) / kWarps + 31) & ~31;
     const int lo = min(warp * seg, n_local), hi = min(lo + seg, n_local);
@@ -179,7 +482,7 @@ __device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, cons
         const int i = i0 + lane;
         uint32_t mk = 0;
         const bool in = i < hi;
-        if (in) mk = float_to_key(vals[i]) & th.mask;
+        if (in) mk = float_to_key(row.at(i)) & th.mask;
         gt += __popc(__ballot_sync(0xffffffffu, in && mk > th.prefix));
         eq += __popc(__ballot_sync(0xffffffffu, in && mk == th.prefix));
     }
@@ -202,22 +505,32 @@ __device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, cons
     uint32_t gt_before = s.wcnt[warp], eq_before = s.wcnt[kWarps + warp];
     if (C > 1) {
         cl.sync();
-        for (int p = 0; p < rank; ++p) {
-            const uint32_t *pm = cl.map_shared_rank(s.misc, p);
-            gt_before += pm[4];
-            eq_before += pm[5];
+        // lane p reads rank p's totals, so the remote reads overlap
+        uint32_t g = 0, e = 0;
+        if (lane < rank) {
+            const uint32_t *pm = cl.map_shared_rank(s.misc, lane);
+            g = pm[4];
+            e = pm[5];
         }
+        gt_before += __reduce_add_sync(0xffffffffu, g);
+        eq_before += __reduce_add_sync(0xffffffffu, e);
     }
     for (int i0 = lo; i0 < hi; i0 += 32) {
         const int i = i0 + lane;
         uint32_t mk = 0;
         const bool in = i < hi;
-        if (in) mk = float_to_key(vals[i]) & th.mask;
+        int at = 0;
+        if (in) {
+            at = row.pos(i);
+            mk = float_to_key(row.vals[at]) & th.mask;
+        }
         const bool is_gt = in && mk > th.prefix, is_eq = in && mk == th.prefix;
         const unsigned bg = __ballot_sync(0xffffffffu, is_gt), be = __ballot_sync(0xffffffffu, is_eq);
         const unsigned below = (1u << lane) - 1u;
-        const uint32_t g = gt_before + __popc(bg & below), e = eq_before + __popc(be & below);
-        if (is_gt || (is_eq && e < th.remaining)) out[g + min(e, th.remaining)] = base + i;
+        const uint32_t gi = gt_before + __popc(bg & below), e = eq_before + __popc(be & below);
+        const bool keep = is_gt || (is_eq && e < th.remaining);
+        const int t = (int)(gi + min(e, th.remaining));
+        if (keep) out[t] = base + at;
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
@@ -270,8 +583,22 @@ __device__ int merge_exact(const Cand *cand, int slots, int m, Cand *surv)
 // The lists together hold every member of the top-m, and `hist` counts the listed edges per cosine
 // bin: the highest bin b with at least m listed edges in bins >= b bounds the m-th largest from
 // below, so only edges with e >= b / kCandBins need ranking.
-__device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chunks, int m,
-                                 Cand *surv, int *ns_sh, int bar_id, int wg, int *nbr_idx, float *nbr_e)
+// The final list also goes, as (position, decay factor over all rounds), into slots
+// [slot0, slot0 + m) of the nb_j / nb_f arrays of the CTAs of the cluster that hold the row (slots past the listed
+// edges get position -1).
+struct PushLists {
+    int C;          // cluster size
+    int R;          // ranks 0 .. R-1 receive the lists
+    int *nb_j;
+    float *nb_f;
+    int slot0;
+    float lambda;
+    int T;
+};
+
+__device__ void merge_neighbours(cg::cluster_group &cl, const Cand *cand, const uint32_t *hist,
+                                 int chunks, int m, Cand *surv, int *ns_sh, int bar_id, int wg,
+                                 int *nbr_idx, float *nbr_e, const PushLists &push)
 {
     const int lane = threadIdx.x & 31;
     constexpr int kPer = kCandBins / 32;
@@ -347,8 +674,18 @@ __device__ void merge_neighbours(const Cand *cand, const uint32_t *hist, int chu
         if (rank < m) {
             nbr_idx[rank] = me.j;
             nbr_e[rank] = me.e;
+            const float f = 1.0f - push.lambda * fmaxf(me.e, 0.f);
+            float pw = f;
+            for (int t = 1; t < push.T; ++t) pw *= f;
+            for (int p = 0; p < push.R; ++p) {
+                (push.C > 1 ? cl.map_shared_rank(push.nb_j, p) : push.nb_j)[push.slot0 + rank] = me.j;
+                (push.C > 1 ? cl.map_shared_rank(push.nb_f, p) : push.nb_f)[push.slot0 + rank] = pw;
+            }
         }
     }
+    for (int u = ns + wg * 32 + lane; u < m; u += 128)
+        for (int p = 0; p < push.R; ++p)
+            (push.C > 1 ? cl.map_shared_rank(push.nb_j, p) : push.nb_j)[push.slot0 + u] = -1;
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // the list may be reused
 }
 
@@ -531,8 +868,11 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
     const int n_local = max(0, min(a.chunk, N - base));
     float *vals = s.vals + a.halo;
     float *row_s = a.s + (long long)unit * N;
+    PhaseClock pc(threadIdx.x == 0 && rank == 0);
+    pc.mark();
     if (a.wait_prior) pdl_wait();
     pdl_launch_dependents();
+    pc.mark();
     if (a.zero)
         for (int i = rank * kThreads + tid; i < a.zero_words; i += C * kThreads)
             a.zero[(long long)unit * a.zero_words + i] = 0u;
@@ -572,22 +912,31 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
         load_chunk(row_s, base, 0, n_local, N, vals, 0.f);
     }
     __syncthreads();
+    pc.mark();
     if (a.k > 0) {
         int *out = a.src_out + (long long)unit * a.k;
         const bool done = bounded && cluster_topk_bounded(cl, C, rank, s, vals, n_local, base, a.k, hc0, hc1, out);
         if (!done) {
-            const Threshold th = cluster_kth(cl, C, rank, s, vals, n_local, (uint32_t)a.k);
-            cluster_emit_sorted(cl, C, rank, s, vals, n_local, base, th, out);
+            const RowView row{vals, nullptr, n_local};
+            const Threshold th = cluster_kth(cl, C, rank, s, row, (uint32_t)a.k);
+            cluster_emit_sorted(cl, C, rank, s, row, base, th, out);
         }
     }
+    pc.mark();
     if (C > 1) cl.sync();      // no CTA leaves while its shared memory may still be read
+    pc.mark();
+    pc.flush(3);
 }
 
 struct FinishArgs {
     Dims d;
-    int C, chunk;
+    int C;                     // CTAs per cluster (one cluster per unit)
+    int R;                     // ranks 0 .. R-1 hold a chunk of the row each: 1 (the others only
+                               // merge neighbour lists and gather) or C
+    int chunk, halo;
     int unit0;
-    float *s;                  // [units][N] scores (decayed in place when has_graph)
+    const float *a;            // optional [units][N]: attention mass to pool into the scores first
+    float *s;                  // [units][N] scores: read unless pooling; written when pooling or decaying
     int *nbr_idx;              // [units][K_src][m] neighbour lists (has_graph); written when merging
     float *nbr_e;              // [units][K_src][m] their cosines
     int has_graph;             // apply the decay rounds
@@ -603,68 +952,239 @@ struct FinishArgs {
     int wait_prior;            // launched with programmatic stream serialization
 };
 
+// Chunk [base, base + n_local) of a unit's scores into shared memory; returns `vals` with
+// vals[i] = score of element base + i.  With `row_a` the scores are the attention mass max-pooled
+// over [j - half, j + half] (positions outside the row ignored): the raw values are staged first
+// and the pooled value of element i replaces a slot at or below raw slot i, in rounds whose
+// inputs are all read before any is overwritten (element i reads raw slots i .. i + 2 half, so a
+// later round never needs what an earlier one has replaced).  Global reads are 16-byte loads; the
+// staging offset inside `buf` (16-byte aligned, chunk + 2 half + 8 words) is chosen so that the
+// returned values sit at the same offset modulo 16 bytes as the elements of the global row.
+// Ends with the CTA synchronised.
+__device__ float *load_pool_chunk(const float *row_a, const float *row_s, int base, int n_local,
+                                  int N, int half, float *buf)
+{
+    const int tid = threadIdx.x;
+    const float *row = row_a ? row_a : row_s;
+    const int h = row_a ? half : 0;
+    const int j0 = base - h, j1 = base + n_local + h;          // staged span, row positions
+    const int lo = max(j0, 0), hi = min(j1, N);
+    const int e2 = (4 - (h & 3)) & 3;                          // pooled element i goes to slot i - e2
+    const int gcls = (int)((reinterpret_cast<uintptr_t>(row + lo) >> 2) & 3);
+    int pad = (gcls - (lo - j0)) & 3;
+    while (pad < e2) pad += 4;
+    float *dst = buf + pad;                                    // dst[j - j0] = row[j]
+    if (n_local > 0) {
+        for (int j = j0 + tid; j < lo; j += kThreads) dst[j - j0] = -INFINITY;
+        for (int j = max(hi, j0) + tid; j < j1; j += kThreads) dst[j - j0] = -INFINITY;
+        const int head = min(hi - lo, (4 - gcls) & 3);
+        if (tid < head) dst[lo + tid - j0] = __ldcg(row + lo + tid);
+        const int v0 = lo + head, nv = (hi - v0) >> 2;
+        const float4 *rv = reinterpret_cast<const float4 *>(row + v0);
+        float4 *dv = reinterpret_cast<float4 *>(dst + (v0 - j0));
+        for (int i0 = tid; i0 < nv; i0 += 8 * kThreads) {
+            float4 r[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (i0 + k * kThreads < nv) r[k] = __ldcg(rv + i0 + k * kThreads);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (i0 + k * kThreads < nv) dv[i0 + k * kThreads] = r[k];
+        }
+        const int t0 = v0 + 4 * nv;
+        if (tid < hi - t0) dst[t0 + tid - j0] = __ldcg(row + t0 + tid);
+    }
+    __syncthreads();
+    if (h == 0) return dst;
+    for (int r0 = 0; r0 < n_local; r0 += 8 * kThreads) {
+        float pooled[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = r0 + q * kThreads + tid;
+            pooled[q] = 0.f;
+            if (i < n_local) {
+                float best = dst[i];
+                for (int t = 1; t <= 2 * h; ++t) best = fmaxf(best, dst[i + t]);
+                pooled[q] = best;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = r0 + q * kThreads + tid;
+            if (i < n_local) dst[i - e2] = pooled[q];
+        }
+        __syncthreads();
+    }
+    return dst - e2;
+}
+
+// row[i] = vals[i] for i < n: 16-byte stores where the two sides share their offset modulo 16 bytes.
+__device__ void store_chunk(float *row, const float *vals, int n)
+{
+    const int tid = threadIdx.x;
+    const uintptr_t g = reinterpret_cast<uintptr_t>(row), sm = reinterpret_cast<uintptr_t>(vals);
+    if (((g ^ sm) & 15) != 0) {
+        for (int i = tid; i < n; i += kThreads) row[i] = vals[i];
+        return;
+    }
+    const int head = min(n, (int)((4 - ((g >> 2) & 3)) & 3));
+    if (tid < head) row[tid] = vals[tid];
+    const int nv = (n - head) >> 2;
+    float4 *rv = reinterpret_cast<float4 *>(row + head);
+    const float4 *sv = reinterpret_cast<const float4 *>(vals + head);
+    for (int i = tid; i < nv; i += kThreads) rv[i] = sv[i];
+    const int t0 = head + 4 * nv;
+    if (tid < n - t0) row[t0 + tid] = vals[t0 + tid];
+}
+
+// Eq. 5 on the chunk in shared memory: the unit's lists are in s.nb_j / s.nb_f as (position,
+// factor over all rounds).  A position that only one listed edge points to (counted per slot of a
+// small table, so a slot shared with another position counts as contested) takes its factor at
+// once; the contested ones are applied by one warp, source after source (a source's neighbours are
+// distinct), so that overlapping neighbourhoods multiply in a fixed order.  Uses s.fine as
+// scratch.  Ends with the CTA synchronised.
+__device__ void apply_lists(const Smem &s, float *vals, int base, int n_local, int K_src, int m)
+{
+    const int tid = threadIdx.x;
+    const int pairs = K_src * m;                           // <= kStage, so K_src <= kStage
+    uint32_t *cnt = s.fine;                                // [4096] edges per table slot
+    uint32_t *src_mask = s.fine + 4096;                    // [kStage / 32] sources with a contested edge
+    for (int i = tid; i < 4096 + kStage / 32; i += kThreads) cnt[i] = 0u;
+    __syncthreads();
+    for (int p = tid; p < pairs; p += kThreads) {
+        const int j = s.nb_j[p] - base;
+        if (j >= 0 && j < n_local) atomicAdd(&cnt[j & 4095], 1u);
+    }
+    __syncthreads();
+    for (int p = tid; p < pairs; p += kThreads) {
+        const int j = s.nb_j[p] - base;
+        if (j >= 0 && j < n_local) {
+            if (cnt[j & 4095] == 1u) {
+                vals[j] *= s.nb_f[p];
+            } else {
+                const int q = p / m;
+                atomicOr(&src_mask[q >> 5], 1u << (q & 31));
+            }
+        }
+    }
+    __syncthreads();
+    if (tid < 32) {
+        for (int w = 0; w * 32 < K_src; ++w) {
+            uint32_t mask = src_mask[w];
+            while (mask) {
+                const int q = w * 32 + __ffs(mask) - 1;
+                mask &= mask - 1;
+                for (int u = tid; u < m; u += 32) {
+                    const int j = s.nb_j[q * m + u] - base;
+                    if (j >= 0 && j < n_local && cnt[j & 4095] != 1u) vals[j] *= s.nb_f[q * m + u];
+                }
+                __syncwarp();
+            }
+        }
+    }
+    __syncthreads();
+}
+
 // grid = units * C CTAs in clusters of C; block kThreads.
 __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
 {
     extern __shared__ __align__(16) uint8_t cs_smem[];
     cg::cluster_group cl = cg::this_cluster();
     const Dims &d = a.d;
-    const int C = a.C, rank = C > 1 ? (int)cl.block_rank() : 0;
+    const int C = a.C, R = a.R, rank = C > 1 ? (int)cl.block_rank() : 0;
     const int unit = a.unit0 + blockIdx.x / C;
     const Smem s = carve(cs_smem, 0);
     const int N = d.N, tid = threadIdx.x;
+    const bool holds = rank < R;                           // this CTA keeps a chunk of the row
     const int base = rank * a.chunk;
-    const int n_local = max(0, min(a.chunk, N - base));
+    const int n_local = holds ? max(0, min(a.chunk, N - base)) : 0;
     float *vals = s.vals;
     float *row_s = a.s + (long long)unit * N;
+    PhaseClock pc(tid == 0);
+    pc.mark();
     if (a.wait_prior) pdl_wait();
     pdl_launch_dependents();
-    load_chunk(row_s, base, 0, n_local, N, vals, 0.f);
-    __syncthreads();
-
-    if (a.has_graph && a.merge) {
-        // Eq. 3: the four warps of group g of rank r merge sources (g + kMergeWarps * t) * C + r
-        const int warp = tid >> 5, grp = warp >> 2, wg = warp & 3;
-        Cand *surv = reinterpret_cast<Cand *>(s.st_idx) + grp * kSurvCap;
-        int *ns_sh = reinterpret_cast<int *>(s.misc) + 8 + grp;
-        for (int src = grp * C + rank; src < d.K_src; src += kMergeWarps * C) {
-            const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
-            merge_neighbours(a.cand + slot * kCandCap,
-                             a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
-                             a.cand_chunks, d.m, surv, ns_sh, 1 + grp, wg,
-                             a.nbr_idx + ((long long)unit * d.K_src + src) * d.m,
-                             a.nbr_e + ((long long)unit * d.K_src + src) * d.m);
-        }
-        __threadfence();
-        if (C > 1) cl.sync(); else __syncthreads();
-    }
-
-    if (a.has_graph) {
-        // Eq. 5 over the fixed graph: source after source (a source's neighbours are distinct, so
-        // one source is applied by parallel threads), the T rounds folded into a power.
-        const int *ni = a.nbr_idx + (long long)unit * d.K_src * d.m;
-        const float *ne = a.nbr_e + (long long)unit * d.K_src * d.m;
-        const int per = d.m <= kStage ? kStage / d.m : 0;      // sources staged together
-        if (per > 0) {
-            for (int src0 = 0; src0 < d.K_src; src0 += per) {
-                const int ns = min(per, d.K_src - src0);
-                for (int i = tid; i < ns * d.m; i += kThreads) {
-                    const float f = 1.0f - d.lambda * fmaxf(__ldcg(ne + src0 * d.m + i), 0.f);
-                    float pw = f;
-                    for (int t = 1; t < d.T; ++t) pw *= f;
-                    s.st_idx[i] = __ldcg(ni + src0 * d.m + i) - base;
-                    s.st_f[i] = pw;
-                }
-                __syncthreads();
-                for (int q = 0; q < ns; ++q) {
-                    for (int u = tid; u < d.m; u += kThreads) {
-                        const int j = s.st_idx[q * d.m + u];
-                        if (j >= 0 && j < n_local) vals[j] *= s.st_f[q * d.m + u];
+    pc.mark();
+    const int b = unit / d.hkv, h = unit % d.hkv;
+    const long long row_bytes = (long long)kHeadDim * a.elem_bytes;
+    const int rows_out = d.B + d.W;
+    const int vpr = (int)(row_bytes >> 4);                 // 16-byte pieces per row
+    const unsigned char *k0 = a.K ? a.K + (b * d.ks[0] + h * d.ks[1]) * a.elem_bytes : nullptr;
+    const unsigned char *v0 = a.V ? a.V + (b * d.vs[0] + h * d.vs[1]) * a.elem_bytes : nullptr;
+    unsigned char *k_out = a.K_out ? a.K_out + (long long)unit * rows_out * row_bytes : nullptr;
+    unsigned char *v_out = a.V_out ? a.V_out + (long long)unit * rows_out * row_bytes : nullptr;
+    const long long k_stride = d.ks[2] * a.elem_bytes, v_stride = d.vs[2] * a.elem_bytes;
+    // copies the 16-byte pieces [p0, p1) of output rows [t0, ...): piece p is (row t0 + p / (2 vpr),
+    // K or V, column piece); `src_of(t)` gives the input row.  Four pieces in flight per thread.
+    auto copy_rows = [&](int t0, long long n_pieces, auto src_of) {
+        const long long stride = (long long)C * kThreads;
+        for (long long p0 = (long long)rank * kThreads + tid; p0 < n_pieces; p0 += 4 * stride) {
+            uint4 v[4];
+            unsigned char *dst[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const long long p = p0 + u * stride;
+                dst[u] = nullptr;
+                if (p < n_pieces) {
+                    const int t = t0 + (int)(p / (2 * vpr)), pp = (int)(p % (2 * vpr));
+                    const bool is_v = pp >= vpr;
+                    const int c = is_v ? pp - vpr : pp;
+                    const unsigned char *in = is_v ? v0 : k0;
+                    if (in) {
+                        v[u] = *reinterpret_cast<const uint4 *>(in + src_of(t) * (is_v ? v_stride : k_stride) + c * 16);
+                        dst[u] = (is_v ? v_out : k_out) + (long long)t * row_bytes + c * 16;
                     }
-                    __syncthreads();
                 }
             }
-        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (dst[u]) *reinterpret_cast<uint4 *>(dst[u]) = v[u];
+        }
+    };
+    const bool gathers = a.do_select && (a.K || a.V);
+    if (holds)
+        vals = load_pool_chunk(a.a ? a.a + (long long)unit * N : nullptr, row_s, base, n_local, N, a.halo, s.vals);
+    pc.mark();
+
+    if (a.has_graph) {
+        int *ni = a.nbr_idx + (long long)unit * d.K_src * d.m;
+        float *ne = a.nbr_e + (long long)unit * d.K_src * d.m;
+        const int pairs = d.K_src * d.m;
+        if (pairs <= kStage) {
+            // Eq. 3, then Eq. 5 over the fixed graph with the T rounds folded into a power: the
+            // CTAs that hold the row get the unit's lists as (position, factor) in shared memory
+            if (a.merge) {
+                // the four warps of group g of merging rank r take sources (g + kMergeWarps * t) * M + r;
+                // a first CTA that holds the whole row leaves the merging to the others
+                const int warp = tid >> 5, grp = warp >> 2, wg = warp & 3;
+                Cand *surv = reinterpret_cast<Cand *>(s.st_idx) + grp * kSurvCap;
+                int *ns_sh = reinterpret_cast<int *>(s.misc) + 8 + grp;
+                const bool spare_first = R == 1 && C > 1;
+                const int M = spare_first ? C - 1 : C, mr = spare_first ? rank - 1 : rank;
+                for (int src = grp * M + mr; mr >= 0 && src < d.K_src; src += kMergeWarps * M) {
+                    const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
+                    const PushLists push{C, R, s.nb_j, s.nb_f, src * d.m, d.lambda, d.T};
+                    merge_neighbours(cl, a.cand + slot * kCandCap,
+                                     a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
+                                     a.cand_chunks, d.m, surv, ns_sh, 1 + grp, wg, ni + src * d.m,
+                                     ne + src * d.m, push);
+                }
+                pc.mark();
+                if (C > 1) cl.sync(); else __syncthreads();       // every list has arrived
+                pc.mark();
+            } else if (holds) {
+                for (int i = tid; i < pairs; i += kThreads) {
+                    const float f = 1.0f - d.lambda * fmaxf(__ldcg(ne + i), 0.f);
+                    float pw = f;
+                    for (int t = 1; t < d.T; ++t) pw *= f;
+                    s.nb_j[i] = __ldcg(ni + i);
+                    s.nb_f[i] = pw;
+                }
+                __syncthreads();
+            }
+            if (holds) apply_lists(s, vals, base, n_local, d.K_src, d.m);
+        } else if (holds) {
             for (int src = 0; src < d.K_src; ++src) {
                 for (int u = tid; u < d.m; u += kThreads) {
                     const int j = ni[src * d.m + u] - base;
@@ -678,54 +1198,43 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
                 __syncthreads();
             }
         }
-        for (int i = tid; i < n_local; i += kThreads) row_s[base + i] = vals[i];
     }
+    pc.mark();
+    // the window rows do not depend on the selection (their loads return while the scores are stored)
+    if (gathers) copy_rows(d.B, (long long)d.W * 2 * vpr, [&](int t) { return (long long)(N + (t - d.B)); });
+    if ((a.a || a.has_graph) && holds) store_chunk(row_s + base, vals, n_local);
+    pc.mark();
 
     if (a.do_select) {
         int *idx = a.idx_out + (long long)unit * d.B;
-        const Threshold th = cluster_kth(cl, C, rank, s, vals, n_local, (uint32_t)d.B);
-        cluster_emit_sorted(cl, C, rank, s, vals, n_local, base, th, idx);
+        if (holds) {
+            // rank only the elements that reach a lower bound of the B-th largest, where one is at hand
+            // (the staging arrays of the lists are free by now)
+            int *list = s.st_idx;
+            // (a short chunk is ranked whole: the passes that list candidates would cost more,
+            // and a budget above a sixteenth of the chunk leaves too many to gain anything)
+            const bool sparse = (long long)d.B * 16 <= a.chunk;
+            const int n_c = a.chunk >= 4 * kStage && sparse
+                                ? filter_candidates(s, vals, n_local, (uint32_t)d.B, list, 4 * kStage) : -1;
+            pc.mark();
+            const RowView row{vals, n_c >= 0 ? list : nullptr, n_c >= 0 ? n_c : n_local};
+            // a sparse selection takes the one-pass search, a dense one the digit-by-digit search
+            // (its threshold bin would hold too many elements to rank by counting)
+            const Threshold th = sparse ? cluster_kth_fine(cl, R, rank, s, row, base, (uint32_t)d.B, pc)
+                                        : cluster_kth(cl, R, rank, s, row, (uint32_t)d.B);
+            cluster_emit_sorted(cl, R, rank, s, row, base, th, idx);
+        }
+        pc.mark();
         __threadfence();
         if (C > 1) cl.sync(); else __syncthreads();
-        // gather: the cluster's threads share the 16-byte pieces of the B + W output rows
-        if (a.K || a.V) {
-            const int vec_per_row = kHeadDim * a.elem_bytes / 16;
-            const int rows_out = d.B + d.W;
-            const long long row_bytes = (long long)kHeadDim * a.elem_bytes;
-            const int b = unit / d.hkv, h = unit % d.hkv;
-            const long long total = (long long)rows_out * vec_per_row;
-            const long long stride = (long long)C * kThreads;
-            for (long long p0 = (long long)rank * kThreads + tid; p0 < total; p0 += 4 * stride) {
-                uint4 kv[4], vv[4];
-                long long dst[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const long long p = p0 + u * stride;
-                    dst[u] = -1;
-                    if (p < total) {
-                        const int c = (int)(p % vec_per_row);
-                        const int t = (int)(p / vec_per_row);
-                        const int src_row = t < d.B ? __ldcg(idx + t) : N + (t - d.B);
-                        dst[u] = ((long long)unit * rows_out + t) * row_bytes + c * 16;
-                        if (a.K)
-                            kv[u] = *reinterpret_cast<const uint4 *>(
-                                a.K + (b * d.ks[0] + h * d.ks[1] + src_row * d.ks[2]) * a.elem_bytes + c * 16);
-                        if (a.V)
-                            vv[u] = *reinterpret_cast<const uint4 *>(
-                                a.V + (b * d.vs[0] + h * d.vs[1] + src_row * d.vs[2]) * a.elem_bytes + c * 16);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (dst[u] >= 0) {
-                        if (a.K) *reinterpret_cast<uint4 *>(a.K_out + dst[u]) = kv[u];
-                        if (a.V) *reinterpret_cast<uint4 *>(a.V_out + dst[u]) = vv[u];
-                    }
-                }
-            }
-        }
+        pc.mark();
+        // gather: the cluster's threads share the 16-byte pieces of the B kept rows
+        if (gathers) copy_rows(0, (long long)d.B * 2 * vpr, [&](int t) { return (long long)__ldcg(idx + t); });
     }
+    pc.mark();
     if (C > 1) cl.sync();      // no CTA leaves while its shared memory may still be read
+    pc.mark();
+    pc.flush(rank == 0 ? 4 : 6);      // the first CTA of a cluster and the others apart
 }
 
 }  // namespace cs

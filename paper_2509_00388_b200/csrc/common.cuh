@@ -89,6 +89,45 @@ __device__ __forceinline__ void pdl_wait()
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// ---- optional phase timing (build with -DGRAPHKV_PHASE_TIMING) --------------------------------
+// One thread per CTA stamps %globaltimer at phase boundaries; at the end of the kernel the
+// differences are added into per-kernel tables that graphkv_phase_timing_read copies out.  In the
+// normal build the marks compile to nothing.
+constexpr int kPhaseKernels = 8, kPhaseSlots = 24;
+#ifdef GRAPHKV_PHASE_TIMING
+__device__ unsigned long long g_phase_sum[kPhaseKernels][kPhaseSlots];
+__device__ unsigned long long g_phase_max[kPhaseKernels][kPhaseSlots];
+__device__ unsigned long long g_phase_cnt[kPhaseKernels];
+struct PhaseClock {
+    unsigned long long t[kPhaseSlots];
+    int n;
+    bool on;
+    __device__ explicit PhaseClock(bool o) : n(0), on(o) {}
+    __device__ __forceinline__ void mark()
+    {
+        if (on && n < kPhaseSlots) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t[n++]));
+    }
+    // slot 0: first to last mark; slot i: mark i-1 to mark i
+    __device__ void flush(int k)
+    {
+        if (!on || n < 2) return;
+        for (int i = 1; i < n; ++i) {
+            atomicAdd(&g_phase_sum[k][i], t[i] - t[i - 1]);
+            atomicMax(&g_phase_max[k][i], t[i] - t[i - 1]);
+        }
+        atomicAdd(&g_phase_sum[k][0], t[n - 1] - t[0]);
+        atomicMax(&g_phase_max[k][0], t[n - 1] - t[0]);
+        atomicAdd(&g_phase_cnt[k], 1ull);
+    }
+};
+#else
+struct PhaseClock {
+    __device__ explicit PhaseClock(bool) {}
+    __device__ __forceinline__ void mark() {}
+    __device__ __forceinline__ void flush(int) {}
+};
+#endif
+
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll

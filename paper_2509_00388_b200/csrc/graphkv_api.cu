@@ -27,6 +27,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t status;      // int status word (256 bytes reserved)
     size_t arrivals;    // stats CTAs done per unit [units] (directly after the status word)
+    size_t arrivals2;   // emit CTAs done per unit [units] (directly after those)
     size_t a_hist;      // histogram of the attention mass [units][2048] (directly after the counters)
     size_t row_c;       // softmax row constants [units][GW]
     size_t part;        // softmax row statistics per key chunk
@@ -38,6 +39,8 @@ struct Layout {
     size_t nbr_e;
     size_t cand;        // per-chunk neighbour candidates [units][K_src][sim_chunks][kCandCap]
     size_t cand_hist;   // [units][K_src][kCandBins]
+    size_t src_cand;    // elements the emit sweep lists for the source selection [units][max_parts][kSrcCap]
+    size_t src_cnt;     // [units][max_parts]
     size_t total;
     int n_stat_chunks;  // key chunks of the SIMT statistics sweep
     int max_parts;      // partial statistics per row the region can hold
@@ -89,6 +92,22 @@ int env_int(const char *name, int dflt)
     return v ? atoi(v) : dflt;
 }
 
+// SMs of the current device (queried once per device).
+int sm_count()
+{
+    static std::mutex mu;
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    std::lock_guard<std::mutex> lk(mu);
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 // Units per launch of a sweep.  By default all units go into one launch: measured on B200, the
 // fixed cost of extra launches outweighs serving the later sweeps of a small group from L2
 // (GRAPHKV_L2_GROUP_MB bounds the keys of a group for experiments).
@@ -106,7 +125,7 @@ int units_per_group(const Dims &d)
 // tile times), with at least min_chunks and at most max_chunks.
 int sweep_chunks(int units, int tiles, int min_chunks, int max_chunks)
 {
-    const int n_sms = 148;
+    const int n_sms = sm_count();
     int best = std::max(1, min_chunks);
     long long best_cost = -1;
     const int hi = std::max(best, std::min(tiles, max_chunks));
@@ -135,7 +154,7 @@ ClusterPlan cluster_plan(const Dims &d)
     // 148 SMs when the rows allow it (two waves of clusters of 8 measured 1.8x slower than one
     // wave of clusters of 4 for 32 rows of 131072)
     while (p.C < cs::kMaxCluster && ceil_div(d.N, p.C) > 4096) p.C *= 2;
-    while (p.C > 1 && d.units * p.C > 148 && ceil_div(d.N, p.C / 2) <= cs::kMaxChunk) p.C /= 2;
+    while (p.C > 1 && d.units * p.C > sm_count() && ceil_div(d.N, p.C / 2) <= cs::kMaxChunk) p.C /= 2;
     p.chunk = (ceil_div(d.N, p.C) + 31) & ~31;
     p.ok = p.chunk <= cs::kMaxChunk && p.halo <= cs::kMaxHalo;
     return p;
@@ -174,6 +193,7 @@ Layout layout_of(const Dims &d)
     l.max_parts = l.n_stat_chunks > 148 ? l.n_stat_chunks : 148;
     l.status = take(kAlign);
     l.arrivals = take((size_t)d.units * sizeof(int));
+    l.arrivals2 = take((size_t)d.units * sizeof(int));
     l.a_hist = take((size_t)d.units * tc::kMassBins * sizeof(uint32_t));
     l.row_c = take((size_t)d.units * d.GW * sizeof(float));
     l.part = take((size_t)d.units * l.max_parts * d.GW * 2 * sizeof(float));
@@ -190,6 +210,9 @@ Layout layout_of(const Dims &d)
     const size_t slots = sp.ok ? (size_t)d.units * d.K_src * sp.chunks : 1;
     l.cand = take(slots * kCandCap * sizeof(Cand));
     l.cand_hist = take((size_t)d.units * (d.K_src > 0 ? d.K_src : 1) * kCandBins * sizeof(uint32_t));
+    const bool tail = d.bf16 && d.K_src > 0 && d.K_src <= tc::kSrcMaxK;
+    l.src_cand = take(tail ? (size_t)d.units * l.max_parts * tc::kSrcCap * sizeof(tc::SrcCand) : kAlign);
+    l.src_cnt = take(tail ? (size_t)d.units * l.max_parts * sizeof(int) : kAlign);
     l.total = off;
     return l;
 }
@@ -382,9 +405,21 @@ bool make_k_tensormap(CUtensorMap *tm, const void *K, const Dims &d, int rows)
 }
 
 
+// What the emit sweep does besides the attention mass: the source nodes of Eq. 2 at its tail
+// (k > 0), words cleared for the kernels that follow, the unit's mass histogram for a pooling
+// kernel that follows.
+struct EmitExtras {
+    int k;
+    int *src_out;
+    uint32_t *zero;
+    int zero_words;
+    bool global_hist;
+};
+
 // Attention mass before pooling, a [units][N], tensor-core path (bf16).
 graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
-                           const __nv_bfloat16 *K, float *a, void *ws, cudaStream_t st)
+                           const __nv_bfloat16 *K, float *a, void *ws, cudaStream_t st,
+                           const EmitExtras &ex)
 {
     CUtensorMap tmK;
     if (!make_k_tensormap(&tmK, K, d, d.L)) return GRAPHKV_ERR_CUDA;
@@ -406,12 +441,19 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
     for (int u0 = 0; u0 < d.units && rc == GRAPHKV_OK; u0 += group) {
         const int nu = std::min(group, d.units - u0);
         const int chunks_s = sweep_chunks(nu, tiles_stats, 1, l.max_parts);
-        const int chunks_e = sweep_chunks(nu, tiles_emit, 1, 1 << 20);
+        const int chunks_e = sweep_chunks(nu, tiles_emit, 1, l.max_parts);
         tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), at<float>(ws, l.row_c), at<int>(ws, l.arrivals), a,
-                           at<uint32_t>(ws, l.a_hist), at<int>(ws, l.status), u0, chunks_s, tiles_stats, chunks_s, stages, 0};
+                           ex.global_hist ? at<uint32_t>(ws, l.a_hist) : nullptr, at<int>(ws, l.status), u0,
+                           chunks_s, tiles_stats, chunks_s, stages, 0,
+                           tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, nullptr}, nullptr, 0, 0};
         tc::ScoreTcArgs ea = sa;
         ea.chunks = chunks_e;
         ea.n_tiles = tiles_emit;
+        ea.src = tc::SourceArgs{ex.k, (d.kp - 1) / 2, ex.src_out, at<tc::SrcCand>(ws, l.src_cand),
+                                at<int>(ws, l.src_cnt), l.max_parts, at<int>(ws, l.arrivals2)};
+        ea.zero = ex.zero;
+        ea.zero_words = ex.zero_words;
+        ea.local_hist = ex.k > 0 ? 1 : 0;
         sa.wait_prior = next_launch_is_dependent();
         rc = launch_ex("score_stats_tc", row_tiles == 1 ? tc::score_stats_tc<1> : tc::score_stats_tc<2>,
                        dim3(chunks_s, nu), dim3(tc::kScoreThreads), smem, st, sa.wait_prior != 0, 1, tmK, sa);
@@ -423,14 +465,20 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
     return rc;
 }
 
+constexpr EmitExtras kPlainEmit{0, nullptr, nullptr, 0, true};
+
+inline bool tc_mass(const __nv_bfloat16 *) { return !env_int("GRAPHKV_FORCE_SIMT", 0); }
+inline bool tc_mass(const float *) { return false; }
+
 inline graphkv_status run_mass(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
-                               const __nv_bfloat16 *K, float *a, void *ws, cudaStream_t st)
+                               const __nv_bfloat16 *K, float *a, void *ws, cudaStream_t st,
+                               const EmitExtras &ex = kPlainEmit)
 {
-    if (env_int("GRAPHKV_FORCE_SIMT", 0)) return run_mass_simt(d, l, Q, K, a, ws, st);
-    return run_mass_tc(d, l, Q, K, a, ws, st);
+    if (!tc_mass(Q)) return run_mass_simt(d, l, Q, K, a, ws, st);
+    return run_mass_tc(d, l, Q, K, a, ws, st, ex);
 }
 inline graphkv_status run_mass(const Dims &d, const Layout &l, const float *Q, const float *K,
-                               float *a, void *ws, cudaStream_t st)
+                               float *a, void *ws, cudaStream_t st, const EmitExtras & = kPlainEmit)
 {
     return run_mass_simt(d, l, Q, K, a, ws, st);
 }
@@ -542,21 +590,44 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *
 
 // Decay rounds (when has_graph) on s in place, then (when do_select) the budget selection and
 // the gather of the compact cache.
-graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, float *s, bool has_graph,
-                          bool merge, bool do_select, const void *K, const void *V, void *K_out, void *V_out,
-                          int *idx_out, void *ws, cudaStream_t st)
+// How the finishing kernel spreads a unit over a cluster: a row of up to kMaxChunk scores is held
+// whole by the first CTA (its selection then needs no exchange between CTAs) and the other CTAs of
+// the cluster only merge neighbour lists and gather; a longer row is split over all C CTAs.
+struct FinishPlan {
+    bool ok;
+    int C, R, chunk;
+};
+
+FinishPlan finish_plan(const Dims &d, int halo)
 {
-    if (!has_graph && !do_select) return GRAPHKV_OK;
+    FinishPlan p{false, 1, 1, 0};
+    if (env_int("GRAPHKV_NO_CLUSTER", 0) || halo > cs::kMaxHalo) return p;
     const ClusterPlan cp = cluster_plan(d);
-    if (cp.ok) {
-        cs::FinishArgs fa{d, cp.C, cp.chunk, 0, s, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e),
+    p.C = p.R = cp.C;
+    p.chunk = cp.chunk;
+    p.ok = p.chunk <= cs::kMaxChunk;
+    return p;
+}
+
+graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const float *a, float *s,
+                          bool has_graph, bool merge, bool do_select, const void *K, const void *V,
+                          void *K_out, void *V_out, int *idx_out, void *ws, cudaStream_t st)
+{
+    if (!has_graph && !do_select && !a) return GRAPHKV_OK;
+    const int halo = a ? (d.kp - 1) / 2 : 0;
+    const FinishPlan fp = finish_plan(d, halo);
+    if (fp.ok && cluster_plan(d).ok) {
+        cs::FinishArgs fa{d, fp.C, fp.R, fp.chunk, halo, 0, a, s, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e),
                           has_graph ? 1 : 0, has_graph && merge ? 1 : 0, at<Cand>(ws, l.cand),
                           at<uint32_t>(ws, l.cand_hist), sim_plan(d, d.bf16 != 0).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
                           static_cast<const unsigned char *>(K), static_cast<const unsigned char *>(V),
                           static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0};
         const char *name = has_graph ? (do_select ? "decay_select_gather" : "decay_rounds") : "select_gather";
-        return launch_cluster(name, cs::finish_kernel, fa, d.units, cp.C, cs::smem_bytes(cp.chunk, 0), st);
+        return launch_cluster(name, cs::finish_kernel, fa, d.units, fp.C, cs::smem_bytes(fp.chunk, halo), st);
     }
+    if (a)
+        GKV_LAUNCH("pool_max", st,
+                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a, s)));
     if (has_graph)
         GKV_LAUNCH("decay_rounds", st,
                    (decay_rounds_kernel<<<d.units, 256, 0, st>>>(d, at<int>(ws, l.nbr_idx),
@@ -609,7 +680,7 @@ graphkv_status do_propagate(const Dims &d, const Layout &l, const T *K, float *s
                                          d.K_src * kCandBins, st);
     if (rc != GRAPHKV_OK || !graph_active(d)) return rc;
     if ((rc = run_graph(d, l, K, src, ws, st)) != GRAPHKV_OK) return rc;
-    return run_finish(d, l, (int)sizeof(T), scores, true, sim_plan(d, sizeof(T) == 2).ok, false,
+    return run_finish(d, l, (int)sizeof(T), nullptr, scores, true, sim_plan(d, sizeof(T) == 2).ok, false,
                       nullptr, nullptr, nullptr, nullptr, nullptr, ws, st);
 }
 
@@ -621,18 +692,32 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
     const bool graph = graph_active(d);
     if (reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
     float *a = d.kp > 1 ? at<float>(ws, l.a) : s;
-    graphkv_status rc = run_mass(d, l, Q, K, a, ws, st);
-    if (rc != GRAPHKV_OK) return rc;
     int *src = at<int>(ws, l.src);
     const bool tc_graph = graph && sim_plan(d, sizeof(T) == 2).ok;
-    // the tensor-core emit sweep leaves a histogram of the attention mass behind
-    const bool have_hist = sizeof(T) == 2 && !env_int("GRAPHKV_FORCE_SIMT", 0);
-    rc = run_pool_sources(d, d.kp > 1 ? a : nullptr, s, graph ? d.K_src : 0, src,
-                          have_hist ? at<uint32_t>(ws, l.a_hist) : nullptr,
-                          tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr, d.K_src * kCandBins, st);
-    if (rc != GRAPHKV_OK) return rc;
+    const int halo = (d.kp - 1) / 2;
+    // The tensor-core emit sweep can pick the sources at its tail and the finishing kernel can pool,
+    // which saves the pooling kernel's launch; measured on B200 the serial tail of the unit's last
+    // emit CTA (about 12 us at 32K keys) costs more than that kernel (10 us), so it is off by default.
+    const bool tail_src = tc_mass(Q) && tc_graph && d.K_src <= tc::kSrcMaxK && env_int("GRAPHKV_TAIL_SOURCES", 0);
+    const bool finish_pools = d.kp > 1 && (tail_src || !graph) && finish_plan(d, halo).ok && cluster_plan(d).ok;
+    graphkv_status rc;
+    if (tail_src || !graph) {
+        const EmitExtras ex{tail_src ? d.K_src : 0, src, tail_src ? at<uint32_t>(ws, l.cand_hist) : nullptr,
+                            tail_src ? d.K_src * kCandBins : 0, false};
+        if ((rc = run_mass(d, l, Q, K, a, ws, st, ex)) != GRAPHKV_OK) return rc;
+        if (d.kp > 1 && !finish_pools &&
+            (rc = run_pool_sources(d, a, s, 0, nullptr, nullptr, nullptr, 0, st)) != GRAPHKV_OK)
+            return rc;
+    } else {
+        if ((rc = run_mass(d, l, Q, K, a, ws, st)) != GRAPHKV_OK) return rc;
+        // the tensor-core emit sweep leaves a histogram of the attention mass behind
+        rc = run_pool_sources(d, d.kp > 1 ? a : nullptr, s, d.K_src, src,
+                              tc_mass(Q) ? at<uint32_t>(ws, l.a_hist) : nullptr,
+                              tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr, d.K_src * kCandBins, st);
+        if (rc != GRAPHKV_OK) return rc;
+    }
     if (graph && (rc = run_graph(d, l, K, src, ws, st)) != GRAPHKV_OK) return rc;
-    return run_finish(d, l, (int)sizeof(T), s, graph, sim_plan(d, sizeof(T) == 2).ok, true, K, V,
+    return run_finish(d, l, (int)sizeof(T), finish_pools ? a : nullptr, s, graph, tc_graph, true, K, V,
                       K_out, V_out, idx_out, ws, st);
 }
 
@@ -765,8 +850,8 @@ graphkv_status graphkv_select_gather(const graphkv_params *params, const float *
     const Layout l = layout_of(d);
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     const int elem = params->dtype == GRAPHKV_BF16 ? 2 : 4;
-    return run_finish(d, l, elem, const_cast<float *>(scores), false, false, true, K, V, K_out, V_out,
-                      idx_out, workspace, static_cast<cudaStream_t>(stream));
+    return run_finish(d, l, elem, nullptr, const_cast<float *>(scores), false, false, true, K, V, K_out,
+                      V_out, idx_out, workspace, static_cast<cudaStream_t>(stream));
 }
 
 graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, const void *K,
@@ -852,6 +937,32 @@ int32_t graphkv_trace_read(graphkv_trace_record *out, int32_t capacity)
     }
     g_trace.clear();
     return n;
+}
+
+int32_t graphkv_phase_timing_read(uint64_t *out)
+{
+#ifdef GRAPHKV_PHASE_TIMING
+    if (!out || cudaDeviceSynchronize() != cudaSuccess) return 0;
+    constexpr size_t n = (size_t)kPhaseKernels * kPhaseSlots;
+    std::vector<unsigned long long> sum(n), mx(n), cnt(kPhaseKernels);
+    if (cudaMemcpyFromSymbol(sum.data(), g_phase_sum, n * 8) != cudaSuccess ||
+        cudaMemcpyFromSymbol(mx.data(), g_phase_max, n * 8) != cudaSuccess ||
+        cudaMemcpyFromSymbol(cnt.data(), g_phase_cnt, kPhaseKernels * 8) != cudaSuccess)
+        return 0;
+    for (size_t i = 0; i < n; ++i) {
+        out[2 * i] = sum[i];
+        out[2 * i + 1] = mx[i];
+    }
+    for (int k = 0; k < kPhaseKernels; ++k) out[2 * n + k] = cnt[k];
+    std::fill(sum.begin(), sum.end(), 0ull);
+    cudaMemcpyToSymbol(g_phase_sum, sum.data(), n * 8);
+    cudaMemcpyToSymbol(g_phase_max, sum.data(), n * 8);
+    cudaMemcpyToSymbol(g_phase_cnt, sum.data(), kPhaseKernels * 8);
+    return 1;
+#else
+    (void)out;
+    return 0;
+#endif
 }
 
 const char *graphkv_status_string(graphkv_status status)

@@ -21,6 +21,7 @@
 // sets share a tile, the two pairs take alternate tiles and four buffers rotate).
 #pragma once
 
+#include "source_select.cuh"
 #include "tc_common.cuh"
 
 namespace graphkv {
@@ -46,6 +47,12 @@ struct ScoreTcArgs {
     int stats_chunks;   // key chunks of the statistics sweep (partials per row)
     int stages;         // shared-memory K tiles in flight
     int wait_prior;     // launched with programmatic stream serialization: wait for the kernels before
+    // emit sweep only: the source nodes of Eq. 2 at its tail (src.k = 0: none), and words to clear
+    // for the kernels that follow
+    SourceArgs src;
+    uint32_t *zero;     // optional [units][zero_words]
+    int zero_words;
+    int local_hist;     // build the per-CTA mass histogram even without a_hist
 };
 
 struct ScoreSmem {
@@ -181,6 +188,8 @@ __global__ void __launch_bounds__(kScoreThreads, 1)
 score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
+    PhaseClock pc(threadIdx.x == 64);
+    pc.mark();
     constexpr int kRowsPad = 128 * kRowTiles;
     constexpr int kBufCols = 128 * kRowTiles;        // TMEM columns per accumulator buffer
     constexpr uint32_t kTmemCols = 512;
@@ -211,9 +220,12 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         stage_q(gen, kRowsPad, d, a.Q, b, h, threadIdx.x - 32, kScoreThreads - 32);
         fence_proxy_async();
     }
+    pc.mark();
     if (a.wait_prior) pdl_wait();
+    pc.mark();
     pdl_launch_dependents();
     __syncthreads();
+    pc.mark();
 
     if (warp == 0) {
         if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b);
@@ -286,6 +298,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             }
         }
         ok = alive;
+        pc.mark();
         // partial p of row r: the sets (of every group) that hold columns of the row's tile
         cta_part[(kRowTiles == 1 ? set : set & 1) * kRowsPad + r] = make_float2(mx, z);
     }
@@ -313,6 +326,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         reinterpret_cast<float2 *>(a.part)[((long long)unit * a.stats_chunks + chunk) * d.GW + r] =
             make_float2(mx, z);
     }
+    pc.mark();
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) *s_flag = atomicAdd(a.arrivals + unit, 1) == a.chunks - 1;
@@ -339,6 +353,8 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         }
         if (threadIdx.x == 0) a.arrivals[unit] = 0;      // ready for the next launch
     }
+    pc.mark();
+    pc.flush(0);
 }
 
 // kColTiles = 1 (G*W <= 128) or 2 (G*W <= 256).  grid (chunks, units of the launch).
@@ -347,6 +363,8 @@ __global__ void __launch_bounds__(kScoreThreads, 1)
 score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
+    PhaseClock pc(threadIdx.x == 64);
+    pc.mark();
     constexpr int kRowsPad = 128 * kColTiles;        // rows of the Q operand (UMMA N)
     constexpr int kBufCols = 128 * kColTiles;
     constexpr uint32_t kTmemCols = 512;
@@ -379,14 +397,24 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         stage_q(gen, kRowsPad, d, a.Q, b, h, threadIdx.x - 32, kScoreThreads - 32);
         fence_proxy_async();
     }
+    pc.mark();
     if (a.wait_prior) pdl_wait();
+    pc.mark();
     pdl_launch_dependents();
-    if (a.a_hist)
+    const bool want_hist = a.a_hist != nullptr || a.local_hist;
+    if (want_hist)
         for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads) mass_hist[i] = 0u;
+    if (a.zero) {
+        // this CTA's share of the unit's words to clear
+        const int per_cta = ceil_div(a.zero_words, a.chunks);
+        for (int i = chunk * per_cta + threadIdx.x; i < min((chunk + 1) * per_cta, a.zero_words); i += kScoreThreads)
+            a.zero[(long long)unit * a.zero_words + i] = 0u;
+    }
     // -c_r of the unit's rows; padding rows contribute 2^-inf = 0
     for (int r = threadIdx.x; r < kRowsPad; r += kScoreThreads)
         row_c[r] = r < d.GW ? -__ldcg(a.row_c + (long long)unit * d.GW + r) : -INFINITY;
     __syncthreads();
+    pc.mark();
 
     if (warp == 0) {
         if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b);
@@ -477,14 +505,15 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
                 const float *x = xchg + xb * kSets * 128 + key_lane;
                 const float aj = kSets == 4 ? (x[0] + x[128]) + (x[256] + x[384]) : x[0] + x[128];
                 a_row[j] = aj;
-                if (a.a_hist) atomicAdd(&mass_hist[float_to_key(aj) >> 21], 1u);
+                if (want_hist) atomicAdd(&mass_hist[float_to_key(aj) >> 21], 1u);
             }
         }
         ok = alive;
+        pc.mark();
     }
     if (!ok && a.status) atomicExch(a.status, (int)GRAPHKV_ERR_TIMEOUT);
     tc_fence_before();
-    __syncthreads();
+    const bool all_ok = __syncthreads_and(ok ? 1 : 0) != 0;
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
@@ -494,6 +523,13 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     if (a.a_hist)
         for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads)
             if (mass_hist[i]) atomicAdd(a.a_hist + (long long)unit * kMassBins + i, mass_hist[i]);
+    pc.mark();
+    // Eq. 2: the unit's source nodes (the stage ring is idle by now and serves as scratch)
+    if (a.src.k > 0 && all_ok)
+        source_select_tail(a.src, d, unit, chunk, a.chunks, t0 * kTileKeys, min(t1 * kTileKeys, d.N),
+                           a.a_out + (long long)unit * d.N, mass_hist, gen + (s.stage0 - s.q));
+    pc.mark();
+    pc.flush(1);
 }
 
 }  // namespace tc

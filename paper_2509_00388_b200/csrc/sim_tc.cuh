@@ -105,6 +105,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     uint2 *queue = reinterpret_cast<uint2 *>(max_bin + (NP / 4) * kSimEpiThreads);  // [kQueueCap][256]
     int *xchg = reinterpret_cast<int *>(gen + (s_tmem - base)) + 2;             // 2 words
 
+    PhaseClock pc(threadIdx.x == 64);
+    pc.mark();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int unit = a.unit0 + blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
     const int chunk = blockIdx.x;
@@ -137,8 +139,10 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         tmem_alloc(s_tmem, 512);
         tmem_relinquish();
     }
+    pc.mark();
     if (a.wait_prior) pdl_wait();
     pdl_launch_dependents();
+    pc.mark();
     // source keys -> swizzled operand rows (rows >= K_src are zero), their positions and norms
     // (16 consecutive threads share a row: the row's squared norm is reduced among them)
     for (int i0 = 0; i0 < NP * 16; i0 += kSimThreads) {
@@ -174,6 +178,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(gen + (s_tmem - base));
     bool ok = true;
+    pc.mark();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -256,6 +261,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             }
         }
         ok = alive;
+        pc.mark();
         // every tile's copies and MMAs are complete once both sets are here: the stage memory is free
         if (!alive && lane == 0) xchg[0] = 0;
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -284,6 +290,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 max_bin[g * kSimEpiThreads + et] = word;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
+            pc.mark();
             const int ew = warp - 2;
             for (int g = ew; g * 4 < d.K_src; g += 8) {
                 uint32_t w8[8];              // this lane's eight threads' bins of sources 4g .. 4g+3
@@ -317,6 +324,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
+            pc.mark();
             // 2. list the edges that reach the threshold bin.  theta is the bin's lower edge brought to
             //    the scale of dot / |k_j|, lowered (the bin index rounds: a cosine a few 1e-8 under
             //    the edge still lands in the bin) so that no edge of the bin is missed.
@@ -356,6 +364,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                         : "memory");
                 }
             }
+            pc.mark();
             const int n_queued = static_cast<int>((qa - q_first) / q_step);
             if (n_queued > kQueueCap) xchg[1] = 1;                    // entries were lost
             for (int k = 0; k < min(n_queued, kQueueCap); ++k) {
@@ -368,6 +377,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                     if (pos < kCandCap) list[c * kCandCap + pos] = Cand{e, j};
                 }
             }
+            pc.mark();
             asm volatile("bar.sync 1, 256;" ::: "memory");
             {
                 const bool lost = xchg[1] != 0;
@@ -415,6 +425,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
             }
+            pc.mark();
             // write the lists out (unused slots marked empty) and count the listed edges per bin
             for (int idx = et; idx < d.K_src * kCandCap; idx += kSimEpiThreads) {
                 const int c = idx / kCandCap, q = idx % kCandCap;
@@ -433,6 +444,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 a.cand[slot * kCandCap + i % kCandCap] = Cand{kCandEmpty, -1};
             }
         }
+        pc.mark();
         tc_fence_before();
     }
     if (!ok && a.status) atomicExch(a.status, (int)GRAPHKV_ERR_TIMEOUT);
@@ -443,6 +455,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
+    pc.mark();
+    pc.flush(2);
 }
 
 }  // namespace tc

@@ -157,6 +157,31 @@ def test_zero_queries_give_constant_scores_and_lowest_indices(gk):
     assert torch.equal(out["idx"], torch.arange(77, dtype=torch.int32).expand(1, 2, 77))
 
 
+def test_tail_source_selection_takes_its_radix_path_on_constant_scores(gk):
+    # all-zero queries make every score equal: the sources are the lowest positions, and the
+    # selection at the tail of the emit sweep must reach them through its search over the pooled
+    # row (its candidate lists overflow); the staged calls pick them with the pooling kernel
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=3000, budget=77, n_q_heads=4, n_kv_heads=2, rounds=1,
+                    topk_nodes=16, neighbors=4)
+    inp = wl.make_inputs(cfg)
+    Qw = torch.zeros_like(inp["Qw"])
+    kw = cfg_kwargs(cfg)
+    old = os.environ.get("GRAPHKV_TAIL_SOURCES")
+    os.environ["GRAPHKV_TAIL_SOURCES"] = "1"
+    try:
+        staged = run_staged(gk, Qw, inp["K"], inp["V"], **kw)
+        fused = run_fused(gk, Qw, inp["K"], inp["V"], **kw)
+    finally:
+        if old is None:
+            os.environ.pop("GRAPHKV_TAIL_SOURCES", None)
+        else:
+            os.environ["GRAPHKV_TAIL_SOURCES"] = old
+    assert torch.equal(staged["src"], torch.arange(16, dtype=torch.int32).expand(1, 2, 16))
+    for name in ("idx", "K_out", "V_out", "scores"):
+        assert torch.equal(staged[name].view(torch.uint8), fused[name].view(torch.uint8)), name
+    assert torch.equal(torch.sort(staged["nbr"], dim=-1).values, torch.sort(fused["nbr"], dim=-1).values)
+
+
 def test_exact_duplicate_keys_tie_break_like_the_oracle(gk):
     # bit-identical keys give bit-identical cosines: the lower index must win on both sides
     cfg = wl.scaled(wl.LLAMA_32K, n_prefix=2000, budget=100, n_q_heads=4, n_kv_heads=1,
@@ -194,10 +219,12 @@ def test_identical_keys_take_the_exact_tie_paths(gk):
 
 @pytest.mark.parametrize("env", [{"GRAPHKV_NO_CLUSTER": "1"}, {"GRAPHKV_FORCE_SIMT": "1"},
                                  {"GRAPHKV_NO_CLUSTER": "1", "GRAPHKV_FORCE_SIMT": "1"},
-                                 {"GRAPHKV_L2_GROUP_MB": "1"}])
+                                 {"GRAPHKV_L2_GROUP_MB": "1"}, {"GRAPHKV_TAIL_SOURCES": "1"},
+                                 {"GRAPHKV_TAIL_SOURCES": "1", "GRAPHKV_NO_CLUSTER": "1"}])
 def test_fallback_kernels_agree_with_the_oracle(gk, env):
     # the generic row kernels (rows too long for a cluster), the SIMT sweeps (fp32 inputs, many
-    # sources or neighbours) and several launch groups, forced here on a case the fast path covers
+    # sources or neighbours), several launch groups, and the source selection at the tail of the
+    # emit sweep with pooling in the finishing kernel, forced here on a case the fast path covers
     cfg = wl.scaled(wl.LLAMA_32K, n_prefix=4500, budget=300, n_q_heads=8, n_kv_heads=2,
                     n_clusters=32, neighbors=8, batch=2)
     old = {k: os.environ.get(k) for k in env}
