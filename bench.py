@@ -6,7 +6,14 @@ on one layer of the Llama-3.1-8B-shaped workload (32 query / 8 KV heads, head_di
 N = 32768 prefix tokens, window 32, budget 512, 16 source nodes, 2 rounds), bf16, synthetic
 seeded inputs.  Metric: context tokens per second per layer, all heads (batch * N / step time).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+The timed region is R blocks of K steps back to back, each block bracketed by CUDA events on the
+launching stream; the step time is the median block divided by K (minimum, maximum and the SM
+clock sampled during the region are reported beside it).  The default run also times the
+131072-token, 4-sequence workload the same way and attaches it as `secondary`.  Workloads with
+several layers (32-layer models, per-layer budgets) step through their layers in order: a step is
+one layer, and the whole-model time is reported too.
 
 Under torchrun (N > 1) every rank runs an independent replica on its own GPU (the path has no
 exchange step); the timed region is bracketed by a barrier and a device synchronise, the step
@@ -33,8 +40,9 @@ from paper_2509_00388_b200 import workloads as wl  # noqa: E402
 
 METRIC = "prefill KV-compress context tokens/sec per layer (all heads)"
 UNIT = "tokens/s"
-ROTATING_SETS = 4          # distinct device copies of the inputs; 4 x 67 MB of K > 126 MB L2
+L2_BYTES = 126e6
 FALLBACK_HBM_GBS = 6650.0
+SECONDARY = "long_128k_batch4"
 
 
 def cfg_kwargs(cfg, layer=0):
@@ -44,9 +52,10 @@ def cfg_kwargs(cfg, layer=0):
 
 
 def config_dict(cfg, extra=None):
-    d = {"workload": cfg.name, "batch": cfg.batch, "n_q_heads": cfg.n_q_heads,
-         "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim, "n_prefix": cfg.n_prefix,
-         "window": cfg.window, "budget": cfg.budget, "pool_kernel": cfg.pool_kernel,
+    d = {"workload": cfg.name, "batch": cfg.batch, "n_layers": cfg.n_layers,
+         "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
+         "n_prefix": cfg.n_prefix, "window": cfg.window, "budget": cfg.budget,
+         "budget_last": cfg.budget_last, "pool_kernel": cfg.pool_kernel,
          "topk_nodes": cfg.topk_nodes, "neighbors": cfg.neighbors, "rounds": cfg.rounds,
          "decay": cfg.decay, "parallelism": "replicas"}
     if extra:
@@ -55,13 +64,17 @@ def config_dict(cfg, extra=None):
 
 
 # ---- algorithmic bytes -------------------------------------------------------------------------
+def mean_budget(cfg) -> float:
+    return sum(cfg.layer_budget(l) for l in range(cfg.n_layers)) / cfg.n_layers
+
+
 def algorithmic_bytes(cfg, kernel: str) -> float:
     """Bytes a kernel must move per launch for one layer of cfg (inputs it has to read once and
     outputs it has to write once; on-chip intermediates are not counted)."""
     e = 2 if cfg.dtype == "bf16" else 4
     units = cfg.batch * cfg.n_kv_heads
     N, L, D, W = cfg.n_prefix, cfg.seq_len, cfg.head_dim, cfg.window
-    B, Ks = cfg.budget, cfg.topk_nodes
+    B, Ks = mean_budget(cfg), cfg.topk_nodes
     m = cfg.neighbors
     k_sweep = units * L * D * e
     q_bytes = cfg.batch * cfg.n_q_heads * W * D * e
@@ -69,7 +82,6 @@ def algorithmic_bytes(cfg, kernel: str) -> float:
     table = {
         "score_stats": k_sweep + q_bytes,
         "score_emit": units * N * D * e + q_bytes + row,
-        "score_fused": k_sweep + q_bytes + row,
         "pool_max": 2 * row,
         "pool_select_sources": 2 * row + 4 * units * Ks,
         "decay_select_gather": 2 * row + 4 * units * B + 4 * units * (B + W) * D * e,
@@ -87,12 +99,11 @@ def algorithmic_bytes(cfg, kernel: str) -> float:
     return 0.0
 
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
-# summarised in profiles/kernels_llama31_8b_32k_ncu_full.md; cold cache.  Only for the workload
-# and kernels that capture covers; anything else reports null.
-NCU_TRAFFIC = {"llama31_8b_32k": {"score_stats_tc": 67.86e6, "score_emit_tc": 67.87e6,
-                                  "pool_select_sources": 1.18e6, "similarity_tc": 67.66e6,
-                                  "decay_select_gather": 4.66e6}}
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum), one ncu capture per
+# kernel inside a running step (caches as the steps before left them); see
+# profiles/kernels_llama31_8b_32k_ncu_warm.md.  Only for the workload and kernels those captures
+# cover and only while the kernels are the ones captured; anything else reports null.
+NCU_TRAFFIC = {}
 
 
 def path_bytes(cfg) -> float:
@@ -103,7 +114,13 @@ def path_bytes(cfg) -> float:
     return float(2 * units * cfg.seq_len * cfg.head_dim * e
                  + cfg.batch * cfg.n_q_heads * cfg.window * cfg.head_dim * e
                  + 12 * units * cfg.n_prefix
-                 + 4 * units * (cfg.budget + cfg.window) * cfg.head_dim * e)
+                 + 4 * units * (mean_budget(cfg) + cfg.window) * cfg.head_dim * e)
+
+
+def one_sweep_bytes(cfg) -> float:
+    """The stricter model: as if the second sweep of K were served on chip."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    return path_bytes(cfg) - cfg.batch * cfg.n_kv_heads * cfg.seq_len * cfg.head_dim * e
 
 
 def measured_peak():
@@ -165,7 +182,7 @@ class ClockSampler:
         reasons = [name for bit, name in self.REASONS.items()
                    if self.mask & bit and name != "gpu_idle"]
         return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(s)}
+                "samples": len(s), "sm_mhz_min": s[0]}
 
 
 def visible_gpu_index(local_rank: int) -> int:
@@ -245,6 +262,160 @@ def run_reference(args, cfg):
 
 
 # ---- our arm -----------------------------------------------------------------------------------
+def input_stats(cfg, inp):
+    """Sanity statistics of a generated input (first sequence, first KV head): the mean cosine of
+    the keys to their head's mean direction, the share of near-duplicate pairs among 4096 sampled
+    neighbours-in-position, and the query norm; a degenerate generator shows up here."""
+    K = inp["K"][0, 0, :min(cfg.n_prefix, 4096)].float()
+    Kn = K / K.norm(dim=1, keepdim=True).clamp_min(1e-12)
+    g = Kn @ Kn[:256].T
+    return {"key_norm_mean": float(K.norm(dim=1).mean()),
+            "cos_mean_to_first_256": float(g.mean()),
+            "cos_above_0.99_share": float((g > 0.99).float().mean()),
+            "query_norm_mean": float(inp["Qw"][0, 0].float().norm(dim=1).mean())}
+
+
+def measure(cfg, gk, dev, world, local, steps, warmup, blocks, with_e2e):
+    """Times cfg on the current device.  Returns a dict of raw measurements."""
+    n_sets_layers = min(cfg.n_layers, 4)          # distinct layers' inputs generated (the rest reuse them)
+    k_bytes = cfg.batch * cfg.n_kv_heads * cfg.seq_len * cfg.head_dim * (2 if cfg.dtype == "bf16" else 4)
+    # distinct device copies of the inputs, so that the first sweep of a step reads HBM: enough
+    # for the keys touched between two uses of a copy to exceed twice the L2
+    copies = max(1, -(-int(2.0 * L2_BYTES) // (k_bytes * n_sets_layers)))
+    host_sets = [wl.make_inputs(cfg, layer=l) for l in range(n_sets_layers)]
+    stats = input_stats(cfg, host_sets[0])
+    host = [{k: v.pin_memory() for k, v in h.items()} for h in host_sets]
+    sets = [{k: v.to(dev).clone() for k, v in h.items()} for _ in range(copies) for h in host]
+    params = [gk.make_params(sets[0]["K"], Qw=sets[0]["Qw"], V=sets[0]["V"], **cfg_kwargs(cfg, l))
+              for l in range(cfg.n_layers)]
+    ws = gk.alloc_workspace(max(params, key=gk.workspace_bytes), dev)
+    bufs = {}                                     # outputs are dense per budget
+    for p in params:
+        if p.budget not in bufs:
+            bufs[p.budget] = gk.alloc_outputs(p, sets[0]["K"], want_scores=False)[:3]
+    torch.cuda.synchronize(dev)
+
+    def step(i):
+        layer = i % cfg.n_layers
+        s = sets[((i // cfg.n_layers) % copies) * n_sets_layers + layer % n_sets_layers]
+        p = params[layer]
+        ko, vo, io = bufs[p.budget]
+        gk.graphkv_compress(p, s["Qw"], s["K"], s["V"], ko, vo, io, None, ws)
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize(dev)
+    assert gk.graphkv_read_status(ws) == gk.OK
+
+    # ---- timed region: `blocks` blocks of `steps` steps, inputs resident in HBM ----
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(blocks + 1)]
+    launches0 = gk.graphkv_launch_count()
+    barrier(world)
+    torch.cuda.synchronize(dev)
+    with ClockSampler(visible_gpu_index(local)) as clocks:
+        evs[0].record()
+        for b in range(blocks):
+            for i in range(steps):
+                step(b * steps + i)
+            evs[b + 1].record()
+        torch.cuda.synchronize(dev)
+    barrier(world)
+    launches = gk.graphkv_launch_count() - launches0
+    per_block = sorted(evs[b].elapsed_time(evs[b + 1]) / steps for b in range(blocks))
+    med = per_block[len(per_block) // 2]
+    res = {"ms_per_step": max_over_ranks(med, world, dev), "ms_min": per_block[0], "ms_max": per_block[-1],
+           "blocks": blocks, "launches": int(launches), "clocks": clocks.summary(),
+           "input_stats": stats, "copies": copies * n_sets_layers, "k_bytes": k_bytes}
+
+    # ---- per-kernel durations: `steps` steps again with event pairs around every launch ----
+    gk.graphkv_trace_enable(True)
+    for i in range(steps):
+        step(i)
+    torch.cuda.synchronize(dev)
+    gk.graphkv_trace_enable(False)
+    per_kernel = defaultdict(list)
+    for name, ms in gk.graphkv_trace_read(steps * 32 + 64):
+        per_kernel[name].append(ms)
+    res["kernels"] = {n: {"launches_per_step": len(v) / steps, "avg_ms": sum(v) / len(v),
+                          "ms_per_step": sum(v) / steps} for n, v in per_kernel.items()}
+
+    if with_e2e:
+        # ---- end to end: host buffers in, compact cache out, copies inside the timed region ----
+        e2e_steps = max(3, min(steps, 50))
+        p = params[0]
+        ko, vo, io = bufs[p.budget]
+        hK = torch.empty(ko.shape, dtype=ko.dtype).pin_memory()
+        hV = torch.empty(vo.shape, dtype=vo.dtype).pin_memory()
+        hI = torch.empty(io.shape, dtype=io.dtype).pin_memory()
+        dst, src = sets[0], host[0]
+
+        # Qw and K are copied to the device (the sweeps read K three times); V stays in pinned host
+        # memory and the gather reads its B+W kept rows per head through the mapping; the compact
+        # cache and the indices are written to pinned host memory by the gather itself.
+        def e2e_step():
+            for k in ("Qw", "K"):
+                dst[k].copy_(src[k], non_blocking=True)
+            gk.graphkv_compress(p, dst["Qw"], dst["K"], src["V"], hK, hV, hI, None, ws)
+
+        for _ in range(2):
+            e2e_step()
+        torch.cuda.synchronize(dev)
+        barrier(world)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        ev1.record()
+        torch.cuda.synchronize(dev)
+        barrier(world)
+        e2e_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / e2e_steps
+        h2d = sum(src[k].numel() * src[k].element_size() for k in ("Qw", "K")) + \
+            hV.numel() * hV.element_size()                      # the rows of V the gather reads
+        d2h = sum(t.numel() * t.element_size() for t in (hK, hV, hI))
+        res["e2e"] = {"value": world * cfg.batch * cfg.n_prefix / (e2e_ms * 1e-3), "unit": UNIT,
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                      "steps": e2e_steps}
+    res["host_inputs"] = host_sets[0]
+    return res
+
+
+def roofline_blocks(cfg, res, peak, peak_kind):
+    """The dominant kernel's roofline entry, the whole path's, and every kernel's."""
+    kernels = res["kernels"]
+    ms_step = res["ms_per_step"]
+    top = max(kernels, key=lambda n: kernels[n]["ms_per_step"])
+    top_bytes = algorithmic_bytes(cfg, top)
+    achieved = top_bytes / (kernels[top]["avg_ms"] * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC.get(cfg.name, {})
+    roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic.get(top),
+                "peak_source": f"{peak_kind} copy bandwidth",
+                "algorithmic_bytes_per_launch": top_bytes,
+                "avg_launch_ms": kernels[top]["avg_ms"],
+                "timing": "CUDA event pairs around every launch, second pass of the same steps"}
+    pb, ob = path_bytes(cfg), one_sweep_bytes(cfg)
+    path = {"bound": "hbm", "algorithmic_bytes_per_step": pb, "achieved": pb / (ms_step * 1e-3) / 1e9,
+            "peak": peak, "unit": "GB/s", "frac": pb / (ms_step * 1e-3) / 1e9 / peak,
+            "frac_of_8tbs": pb / (ms_step * 1e-3) / 1e9 / 8000.0,
+            "one_sweep_model_bytes": ob, "one_sweep_model_frac": ob / (ms_step * 1e-3) / 1e9 / peak,
+            "traffic": sum(traffic.values()) if traffic and set(traffic) >= set(kernels) else None,
+            "ms_x_sm_mhz": ms_step * (res["clocks"].get("sm_mhz") or 0)}
+    per = {n: {"ms_per_step": round(k["ms_per_step"], 5),
+               "algorithmic_bytes": algorithmic_bytes(cfg, n),
+               "achieved": round(algorithmic_bytes(cfg, n) / (k["avg_ms"] * 1e-3) / 1e9, 1),
+               "frac": round(algorithmic_bytes(cfg, n) / (k["avg_ms"] * 1e-3) / 1e9 / peak, 4),
+               "traffic": traffic.get(n)} for n, k in kernels.items()}
+    return roofline, path, per
+
+
+def l2_note(res):
+    mb = res["k_bytes"] / 1e6
+    if res["copies"] == 1:
+        return f"one resident input set: its {mb:.0f} MB of K alone exceed the 126 MB L2"
+    return (f"rotating {res['copies']} resident input sets ({res['copies'] * mb:.0f} MB of K) "
+            f"> 126 MB L2")
+
+
 def run_ours(args, cfg):
     world, rank, local = dist_setup(args.gpus)
     if not torch.cuda.is_available():
@@ -253,109 +424,29 @@ def run_ours(args, cfg):
     gk.lib()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    kw = cfg_kwargs(cfg)
+    peak, peak_kind = measured_peak()
 
-    inp = wl.make_inputs(cfg)
-    host = {k: v.pin_memory() for k, v in inp.items()}
-    sets = []
-    for _ in range(ROTATING_SETS):
-        sets.append({k: v.to(dev, non_blocking=True).clone() for k, v in host.items()})
-    p = gk.make_params(sets[0]["K"], Qw=sets[0]["Qw"], V=sets[0]["V"], **kw)
-    ws = gk.alloc_workspace(p, dev)
-    K_out, V_out, idx, _ = gk.alloc_outputs(p, sets[0]["K"], want_scores=False)
-    torch.cuda.synchronize(dev)
-
-    def step(i):
-        s = sets[i % ROTATING_SETS]
-        gk.graphkv_compress(p, s["Qw"], s["K"], s["V"], K_out, V_out, idx, None, ws)
-
-    for i in range(args.warmup):
-        step(i)
-    torch.cuda.synchronize(dev)
-    assert gk.graphkv_read_status(ws) == gk.OK
-
-    # ---- timed region: K steps, inputs resident in HBM ----
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = gk.graphkv_launch_count()
-    barrier(world)
-    torch.cuda.synchronize(dev)
-    with ClockSampler(visible_gpu_index(local)) as clocks:
-        ev0.record()
-        for i in range(args.steps):
-            step(i)
-        ev1.record()
-        torch.cuda.synchronize(dev)
-    barrier(world)
-    launches = gk.graphkv_launch_count() - launches0
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
-    ms_step = ms_total / args.steps
+    res = measure(cfg, gk, dev, world, local, args.steps, args.warmup, args.blocks, True)
+    ms_step = res["ms_per_step"]
     tokens_per_step = cfg.batch * cfg.n_prefix
     value = world * tokens_per_step / (ms_step * 1e-3)
+    roofline, path, per = roofline_blocks(cfg, res, peak, peak_kind)
+    inp = res.pop("host_inputs")
 
-    # ---- per-kernel durations: the same K steps again with event pairs around every launch ----
-    gk.graphkv_trace_enable(True)
-    for i in range(args.steps):
-        step(i)
-    torch.cuda.synchronize(dev)
-    gk.graphkv_trace_enable(False)
-    per_kernel = defaultdict(list)
-    for name, ms in gk.graphkv_trace_read(args.steps * 32 + 64):
-        per_kernel[name].append(ms)
-    kernels = {n: {"launches_per_step": len(v) / args.steps, "avg_ms": sum(v) / len(v),
-                   "ms_per_step": sum(v) / args.steps} for n, v in per_kernel.items()}
-    top = max(kernels, key=lambda n: kernels[n]["ms_per_step"])
-    peak, peak_kind = measured_peak()
-    top_bytes = algorithmic_bytes(cfg, top)
-    achieved = top_bytes / (kernels[top]["avg_ms"] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC.get(cfg.name, {}).get(top),
-                "peak_source": f"{peak_kind} copy bandwidth",
-                "algorithmic_bytes_per_launch": top_bytes,
-                "avg_launch_ms": kernels[top]["avg_ms"],
-                "timing": "CUDA event pairs around every launch, second pass of the same steps",
-                "whole_path": {"algorithmic_bytes_per_step": path_bytes(cfg),
-                               "achieved_gbs": path_bytes(cfg) / (ms_step * 1e-3) / 1e9,
-                               "frac_of_peak": path_bytes(cfg) / (ms_step * 1e-3) / 1e9 / peak,
-                               "frac_of_8tbs": path_bytes(cfg) / (ms_step * 1e-3) / 1e9 / 8000.0},
-                "kernels": {n: round(k["ms_per_step"], 5) for n, k in kernels.items()},
-                "per_kernel": {n: {"algorithmic_bytes": algorithmic_bytes(cfg, n),
-                                   "achieved_gbs": round(algorithmic_bytes(cfg, n) / (k["avg_ms"] * 1e-3) / 1e9, 1),
-                                   "frac": round(algorithmic_bytes(cfg, n) / (k["avg_ms"] * 1e-3) / 1e9 / peak, 4)}
-                               for n, k in kernels.items()}}
-
-    # ---- end to end: host buffers in, compact cache out, copies inside the timed region ----
-    e2e_steps = max(3, min(args.steps, 50))
-    hK = torch.empty(K_out.shape, dtype=K_out.dtype).pin_memory()
-    hV = torch.empty(V_out.shape, dtype=V_out.dtype).pin_memory()
-    hI = torch.empty(idx.shape, dtype=idx.dtype).pin_memory()
-    dst = sets[0]
-
-    # Qw and K are copied to the device (the sweeps read K three times); V stays in pinned host
-    # memory and the gather reads its B+W kept rows per head through the mapping; the compact
-    # cache and the indices are written to pinned host memory by the gather itself.
-    def e2e_step():
-        for k in ("Qw", "K"):
-            dst[k].copy_(host[k], non_blocking=True)
-        gk.graphkv_compress(p, dst["Qw"], dst["K"], host["V"], hK, hV, hI, None, ws)
-
-    for _ in range(2):
-        e2e_step()
-    torch.cuda.synchronize(dev)
-    barrier(world)
-    ev0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
-    ev1.record()
-    torch.cuda.synchronize(dev)
-    barrier(world)
-    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / e2e_steps
-    h2d = sum(host[k].numel() * host[k].element_size() for k in ("Qw", "K")) + \
-        hV.numel() * hV.element_size()                      # the rows of V the gather reads
-    d2h = sum(t.numel() * t.element_size() for t in (hK, hV, hI))
-    e2e = {"value": world * tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT,
-           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
-           "steps": e2e_steps}
+    secondary = None
+    if world == 1 and not args.no_secondary and cfg.name != SECONDARY:
+        cfg2 = wl.CONFIGS[SECONDARY]
+        torch.cuda.empty_cache()
+        r2 = measure(cfg2, gk, dev, world, local, max(2, args.steps // 20), 3, max(5, args.blocks // 2), False)
+        r2.pop("host_inputs")
+        rf2, path2, per2 = roofline_blocks(cfg2, r2, peak, peak_kind)
+        secondary = {"config": config_dict(cfg2, {"l2": l2_note(r2)}),
+                     "ms_per_step": r2["ms_per_step"], "ms_min": r2["ms_min"], "ms_max": r2["ms_max"],
+                     "blocks": r2["blocks"],
+                     "value": cfg2.batch * cfg2.n_prefix / (r2["ms_per_step"] * 1e-3), "unit": UNIT,
+                     "roofline": rf2, "roofline_path": path2, "roofline_kernels": per2,
+                     "clocks": r2["clocks"], "gpu_launches": r2["launches"],
+                     "input_stats": r2["input_stats"]}
 
     if rank != 0:
         return
@@ -367,13 +458,20 @@ def run_ours(args, cfg):
         cpu = {"value": tokens_per_step / t, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"one full layer of {cfg.name} (all {cfg.n_kv_heads} KV heads), "
                          f"mean of 3 runs, {t:.2f} s each"}
+    extra = {"l2": l2_note(res)}
+    if cfg.n_layers > 1:
+        extra["whole_model_ms"] = ms_step * cfg.n_layers
+        extra["layers"] = f"a step is one layer; the {cfg.n_layers} layers are stepped through in order"
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-            "config": config_dict(cfg, {"l2": f"rotating {ROTATING_SETS} resident input sets "
-                                              f"({ROTATING_SETS * 67} MB of K) > 126 MB L2"}),
-            "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks.summary(), "e2e": e2e,
-            "gpu_launches": int(launches)}
+            "config": config_dict(cfg, extra),
+            "timing": {"blocks": res["blocks"], "steps_per_block": args.steps, "statistic": "median block",
+                       "ms_min": res["ms_min"], "ms_max": res["ms_max"]},
+            "roofline": roofline, "roofline_path": path, "roofline_kernels": per,
+            "cpu_baseline": cpu, "clocks": res["clocks"], "e2e": res["e2e"],
+            "gpu_launches": res["launches"], "input_stats": res["input_stats"],
+            "secondary": secondary}
     print(json.dumps(line))
 
 
@@ -382,12 +480,17 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--blocks", type=int, default=25, help="timed blocks of --steps steps (median reported)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="llama31_8b_32k", choices=list(wl.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's number of sequences")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = wl.CONFIGS[args.workload]
+    if args.batch > 0:
+        cfg = wl.scaled(cfg, batch=args.batch, name=f"{cfg.name}[batch={args.batch}]")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
