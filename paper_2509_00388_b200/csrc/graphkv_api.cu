@@ -92,6 +92,15 @@ int env_int(const char *name, int dflt)
     return v ? atoi(v) : dflt;
 }
 
+// Limit of the device-side waits in clocks: about two seconds, or GRAPHKV_WAIT_CYCLES (tests make
+// a wait run out with a short one).
+long long wait_cycles()
+{
+    const char *v = getenv("GRAPHKV_WAIT_CYCLES");
+    const long long n = v ? atoll(v) : 0;
+    return n > 0 ? n : tc::kWaitCycles;
+}
+
 // SMs of the current device (queried once per device).
 int sm_count()
 {
@@ -445,7 +454,8 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
         tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), at<float>(ws, l.row_c), at<int>(ws, l.arrivals), a,
                            ex.global_hist ? at<uint32_t>(ws, l.a_hist) : nullptr, at<int>(ws, l.status), u0,
                            chunks_s, tiles_stats, chunks_s, stages, 0,
-                           tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, nullptr}, nullptr, 0, 0};
+                           tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, nullptr}, nullptr, 0, 0,
+                           wait_cycles(), env_int("GRAPHKV_DEBUG_WITHHOLD_COMMIT", 0)};
         tc::ScoreTcArgs ea = sa;
         ea.chunks = chunks_e;
         ea.n_tiles = tiles_emit;
@@ -561,7 +571,7 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *
             const int nu = std::min(group, d.units - u0);
             tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(K), src, at<Cand>(ws, l.cand),
                              at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
-                             sp.n_tiles, sp.stages, 0};
+                             sp.n_tiles, sp.stages, 0, wait_cycles()};
             sa.wait_prior = next_launch_is_dependent();
             const dim3 grid(sp.chunks, nu), block(tc::kSimThreads);
             graphkv_status rc;

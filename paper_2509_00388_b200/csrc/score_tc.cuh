@@ -53,6 +53,9 @@ struct ScoreTcArgs {
     uint32_t *zero;     // optional [units][zero_words]
     int zero_words;
     int local_hist;     // build the per-CTA mass histogram even without a_hist
+    long long wait_cycles;   // limit of every wait of the kernel, in clocks
+    int withhold_commit;     // test hook (statistics sweep): the MMA issuer leaves out the arrival that
+                             // announces its first accumulator, so the wait for it runs out
 };
 
 struct ScoreSmem {
@@ -143,13 +146,13 @@ __device__ __forceinline__ uint32_t score_setup(const ScoreSmem &s, uint8_t *gen
 // TMA producer (one thread): key tiles t0+i of (h, b), i in [i_begin, i_end), into the stage ring.
 // The keys are an input of the call, so the producer never waits for the kernels before.
 __device__ __forceinline__ bool score_produce(const ScoreSmem &s, const CUtensorMap *tmK, int stages,
-                                              int t0, int i_begin, int i_end, int h, int b)
+                                              int t0, int i_begin, int i_end, int h, int b, long long lim)
 {
     bool ok = true;
     int issued = i_begin;
     for (int i = i_begin; i < i_end; ++i) {
         const int st = i % stages, ph = (i / stages) & 1;
-        if (!mbar_wait(s.empty0 + 8 * st, ph ^ 1)) { ok = false; break; }
+        if (!mbar_wait(s.empty0 + 8 * st, ph ^ 1, lim)) { ok = false; break; }
         const uint32_t dst = s.stage0 + st * kTileBytes;
         mbar_expect_tx(s.full0 + 8 * st, kTileBytes);
         tma_load_4d(dst, tmK, s.full0 + 8 * st, 0, (t0 + i) * kTileKeys, h, b);
@@ -158,7 +161,7 @@ __device__ __forceinline__ bool score_produce(const ScoreSmem &s, const CUtensor
     }
     if (!ok)        // gave up: let the copies already in flight land before the CTA exits
         for (int i = max(0, issued - stages); i < issued; ++i)
-            mbar_wait(s.full0 + 8 * (i % stages), (i / stages) & 1);
+            mbar_wait(s.full0 + 8 * (i % stages), (i / stages) & 1, lim);
     return ok;
 }
 
@@ -198,6 +201,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     // (four buffers), so that a round of waiting, loading and releasing covers as much arithmetic.
     constexpr int kBufs = 512 / kBufCols, kGroups = 2 / kRowTiles;
     const Dims &d = a.d;
+    const long long lim = a.wait_cycles;
     uint8_t *gen;
     const ScoreSmem s = score_smem_layout(smem_raw, kRowsPad, a.stages, &gen);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -215,7 +219,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols, kEpiWarps / kGroups);
     bool ok = true;
     if (warp == 0) {
-        if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b);
+        if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b, lim);
     } else {
         stage_q(gen, kRowsPad, d, a.Q, b, h, threadIdx.x - 32, kScoreThreads - 32);
         fence_proxy_async();
@@ -228,15 +232,15 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     pc.mark();
 
     if (warp == 0) {
-        if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b);
+        if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b, lim);
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
             for (int i = 0; i < n_local; ++i) {
                 const int st = i % a.stages, ph = (i / a.stages) & 1;
                 const int buf = i % kBufs, bph = (i / kBufs) & 1;
-                if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1)) { ok = false; break; }
-                if (!mbar_wait(s.full0 + 8 * st, ph)) { ok = false; break; }
+                if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1, lim)) { ok = false; break; }
+                if (!mbar_wait(s.full0 + 8 * st, ph, lim)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t kt = s.stage0 + st * kTileBytes;
 #pragma unroll
@@ -250,7 +254,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
                     }
                 }
                 umma_commit(s.empty0 + 8 * st);
-                umma_commit(s.tfull0 + 8 * buf);
+                if (!(a.withhold_commit && i == 0)) umma_commit(s.tfull0 + 8 * buf);
             }
         }
     } else {
@@ -270,7 +274,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         bool alive = true;
         for (int i = grp; i < n_local && alive; i += kGroups) {
             const int buf = i % kBufs, bph = (i / kBufs) & 1;
-            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, bph));
+            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, bph, lim));
             if (!alive) break;
             tc_fence_after();
             uint32_t raw[kSetCols / 32][32];
@@ -375,6 +379,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     constexpr int kBufs = 512 / kBufCols, kGroups = 2 / kColTiles, kSets = 4 / kGroups;
     constexpr int kXchg = 16 / kSets;                // exchange buffers in rotation
     const Dims &d = a.d;
+    const long long lim = a.wait_cycles;
     uint8_t *gen;
     const ScoreSmem s = score_smem_layout(smem_raw, kRowsPad, a.stages, &gen);
     float *row_c = reinterpret_cast<float *>(gen + (s.misc - s.q));      // [kRowsPad]
@@ -392,7 +397,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     const uint32_t tmem_base = score_setup(s, gen, &tmK, a.stages, kTmemCols, kEpiWarps / kGroups);
     bool ok = true;
     if (warp == 0) {
-        if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b);
+        if (lane == 0) ok = score_produce(s, &tmK, a.stages, t0, 0, n_ahead, h, b, lim);
     } else {
         stage_q(gen, kRowsPad, d, a.Q, b, h, threadIdx.x - 32, kScoreThreads - 32);
         fence_proxy_async();
@@ -417,15 +422,15 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     pc.mark();
 
     if (warp == 0) {
-        if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b);
+        if (lane == 0 && ok) ok = score_produce(s, &tmK, a.stages, t0, n_ahead, n_local, h, b, lim);
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(128, n_cols);
             for (int i = 0; i < n_local; ++i) {
                 const int st = i % a.stages, ph = (i / a.stages) & 1;
                 const int buf = i % kBufs, bph = (i / kBufs) & 1;
-                if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1)) { ok = false; break; }
-                if (!mbar_wait(s.full0 + 8 * st, ph)) { ok = false; break; }
+                if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1, lim)) { ok = false; break; }
+                if (!mbar_wait(s.full0 + 8 * st, ph, lim)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t kt = s.stage0 + st * kTileBytes;
 #pragma unroll
@@ -463,7 +468,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         };
         for (int i = grp; i < n_local && alive; i += kGroups) {
             const int buf = i % kBufs;
-            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, (i / kBufs) & 1));
+            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, (i / kBufs) & 1, lim));
             if (!alive) break;
             tc_fence_after();
             auto release = [&]() {
@@ -499,7 +504,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
             __syncwarp();
             if (lane == 0) mbar_arrive(s.xbar0 + 8 * xb);
             if (part != (i / kGroups) % kSets) continue;
-            alive = __all_sync(0xffffffffu, mbar_wait(s.xbar0 + 8 * xb, (i / kXchg) & 1));
+            alive = __all_sync(0xffffffffu, mbar_wait(s.xbar0 + 8 * xb, (i / kXchg) & 1, lim));
             const int j = (t0 + i) * kTileKeys + key_lane;
             if (alive && j < d.N) {
                 const float *x = xchg + xb * kSets * 128 + key_lane;

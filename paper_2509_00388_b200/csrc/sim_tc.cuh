@@ -43,6 +43,7 @@ struct SimTcArgs {
     int n_tiles;           // 128-key tiles per unit
     int stages;
     int wait_prior;        // launched with programmatic stream serialization
+    long long wait_cycles; // limit of every wait of the kernel, in clocks
 };
 
 template <int NP> __host__ __device__ constexpr int sim_tiles_cap() { return 512 / NP; }
@@ -80,6 +81,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     extern __shared__ uint8_t smem_raw[];
     constexpr int kTilesCap = sim_tiles_cap<NP>();
     const Dims &d = a.d;
+    const long long lim = a.wait_cycles;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t s_src = base;
@@ -185,7 +187,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             int issued = n_ahead;
             for (int i = n_ahead; i < n_local; ++i) {
                 const int st = i % a.stages, ph = (i / a.stages) & 1;
-                if (!mbar_wait(s_empty0 + 8 * st, ph ^ 1)) { ok = false; break; }
+                if (!mbar_wait(s_empty0 + 8 * st, ph ^ 1, lim)) { ok = false; break; }
                 const uint32_t dst = s_stage0 + st * kTileBytes;
                 mbar_expect_tx(s_full0 + 8 * st, kTileBytes);
                 tma_load_4d(dst, &tmK, s_full0 + 8 * st, 0, (t0 + i) * kTileKeys, h, b);
@@ -194,14 +196,14 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             }
             if (!ok)        // gave up: let the copies already in flight land before the CTA exits
                 for (int i = max(0, issued - a.stages); i < issued; ++i)
-                    mbar_wait(s_full0 + 8 * (i % a.stages), (i / a.stages) & 1);
+                    mbar_wait(s_full0 + 8 * (i % a.stages), (i / a.stages) & 1, lim);
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, NP);
             for (int i = 0; i < n_local; ++i) {
                 const int st = i % a.stages, ph = (i / a.stages) & 1;
-                if (!mbar_wait(s_full0 + 8 * st, ph)) { ok = false; break; }
+                if (!mbar_wait(s_full0 + 8 * st, ph, lim)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t kt = s_stage0 + st * kTileBytes;
 #pragma unroll
@@ -228,7 +230,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         for (int i = set; i < n_local; i += 2) {
             const int st = i % a.stages, ph = (i / a.stages) & 1;
             float inv = 0.f;
-            if (alive) alive = __all_sync(0xffffffffu, mbar_wait(s_full0 + 8 * st, ph));
+            if (alive) alive = __all_sync(0xffffffffu, mbar_wait(s_full0 + 8 * st, ph, lim));
             if (alive) {
                 // squared norm of this thread's key from the staged tile
                 const uint8_t *tile = gen + (s_stage0 - base) + st * kTileBytes;
@@ -248,7 +250,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 inv_norm[i * 128 + key_lane] = inv;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(s_empty0 + 8 * st);
-                alive = __all_sync(0xffffffffu, mbar_wait(s_done0 + 8 * i, 0));
+                alive = __all_sync(0xffffffffu, mbar_wait(s_done0 + 8 * i, 0, lim));
             }
             if (alive) {
                 tc_fence_after();

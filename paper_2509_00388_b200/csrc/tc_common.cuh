@@ -13,7 +13,7 @@ namespace tc {
 constexpr int kTileKeys = 128;                              // keys per MMA tile (UMMA M or N)
 constexpr int kHalfBytes = kTileKeys * 64 * 2;              // 128 rows x 64 bf16 (one swizzle atom wide)
 constexpr int kTileBytes = 2 * kHalfBytes;                  // 128 keys x 128 dims bf16
-constexpr long long kWaitCycles = 4000000000LL;             // ~2 s at 2 GHz
+constexpr long long kWaitCycles = 4000000000LL;             // default limit of a wait: ~2 s at 2 GHz
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
@@ -50,8 +50,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait for the phase with the given parity to complete.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait for the phase with the given parity to complete: false after `limit` clocks.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit)
 {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
@@ -59,7 +59,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity)) return true;
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
 }
 
