@@ -28,7 +28,10 @@
  *   - Every top-k keeps exactly k items; equal values are ordered lower index first, so results
  *     are deterministic.
  *   - One workspace serves one call at a time: calls sharing a workspace must be ordered on
- *     one stream.
+ *     one stream.  graphkv_score and graphkv_compress clear the status word at its head; a
+ *     workspace whose first use is another call (graphkv_propagate after graphkv_score_knorm,
+ *     graphkv_select_gather alone) must be zero-filled once by its owner for graphkv_read_status
+ *     to mean anything.
  */
 #ifndef GRAPHKV_H_
 #define GRAPHKV_H_
@@ -52,7 +55,13 @@ typedef enum {
 } graphkv_status;
 
 typedef enum { GRAPHKV_BF16 = 0, GRAPHKV_F32 = 1 } graphkv_dtype;
-typedef enum { GRAPHKV_POOL_MAX = 0 } graphkv_pool;
+typedef enum { GRAPHKV_POOL_MAX = 0, GRAPHKV_POOL_AVG = 1 } graphkv_pool;
+/* What a source node sends to its neighbours (Discussion, "Diversity of Graph Signal"): the decay
+ * signal of Eq. 4-5, an enhanced signal (factor 1 + lambda*e), or an evicted signal (the
+ * neighbour's score becomes -inf). */
+typedef enum { GRAPHKV_SIGNAL_DECAY = 0, GRAPHKV_SIGNAL_ENHANCE = 1, GRAPHKV_SIGNAL_EVICT = 2 } graphkv_signal;
+/* Which vectors an edge compares (Discussion, "Exploration of similarity for Graph Edge"). */
+typedef enum { GRAPHKV_TENSOR_K = 0, GRAPHKV_TENSOR_V = 1 } graphkv_tensor;
 
 typedef struct {
     int32_t batch;        /* independent sequences (or any independent units sharing the shape)  */
@@ -62,8 +71,9 @@ typedef struct {
     int32_t seq_len;      /* L = N + W rows present in K and V                                   */
     int32_t window;       /* W >= 1 observation-window rows: queried from, always kept           */
     int32_t budget;       /* B = k_l: prefix tokens kept, 1 <= B <= N; outputs hold B + W rows   */
-    int32_t pool_kernel;  /* odd >= 1 (1 = no pooling); 1-D max pooling of the initial score     */
-    int32_t pool_mode;    /* graphkv_pool                                                        */
+    int32_t pool_kernel;  /* odd >= 1 (1 = no pooling); 1-D pooling of the initial score         */
+    int32_t pool_mode;    /* graphkv_pool: maximum, or mean over pool_kernel positions with zeros
+                             outside the row                                                     */
     int32_t topk_nodes;   /* k of Eq. 2: number of source nodes, 0 <= k <= N (0: no propagation) */
     int32_t neighbors;    /* m of Eq. 3; 0 = adaptive: clamp(floor(N/1000), 1, 32), at most N-1  */
     int32_t rounds;       /* T of Eq. 5, >= 0; 0 = the base method's plain top-B                 */
@@ -72,6 +82,10 @@ typedef struct {
     int64_t q_stride[3];  /* element strides of Qw: batch, head, row                             */
     int64_t k_stride[3];  /* element strides of K: batch, head, token                            */
     int64_t v_stride[3];  /* element strides of V: batch, head, token                            */
+    int32_t signal;       /* graphkv_signal; 0 = the decay signal of Eq. 4-5                     */
+    int32_t reselect;     /* 0: the graph is built once and reused by all T rounds (Algorithm 2);
+                             1: every round re-picks the sources from the current scores and
+                             rebuilds their neighbourhoods (1 + T sweeps of the keys)            */
 } graphkv_params;
 
 /* Bytes of scratch any of the calls below needs for these params; 0 if the params are invalid
@@ -125,6 +139,14 @@ graphkv_status graphkv_score_noalloc(const graphkv_params *params, const void *Q
                                      float *scores, void *stream);
 graphkv_status graphkv_read_status_noalloc(void *stream);
 
+/* Another initial score for step (I): KNorm (Experimental Setup, baseline methods: the L2 norm of
+ * the keys; the cited method keeps the keys of lowest norm).  Writes s_j = 1 / max(||k_j||, 1e-12)
+ * for the prefix keys, scores [batch][n_kv_heads][N] fp32: the ranking of ascending norm, as
+ * positive scores (which the multiplicative decay needs).  One pass over K; no workspace.  Feed
+ * the result to graphkv_propagate and graphkv_select_gather like any other initial score. */
+graphkv_status graphkv_score_knorm(const graphkv_params *params, const void *K, float *scores,
+                                   void *stream);
+
 /* Steps (II)+(III), "Build Graph" and "Decay Signal Propagation" (Eq. 1-5, Algorithms 1-2):
  * sources = top-k of `scores`; e_ij = cosine(k_i, k_j) for each source i and every prefix j != i;
  * N(o_i) = the m largest e_ij; then T times s_j <- s_j * prod_{i: j in N(o_i)} (1 - lambda*max(e_ij,0)).
@@ -135,6 +157,17 @@ graphkv_status graphkv_read_status_noalloc(void *stream);
 graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, float *scores,
                                  int32_t *src_idx_out, void *workspace, size_t workspace_bytes,
                                  void *stream);
+
+/* graphkv_propagate with other edges (Discussion, "Exploration of similarity for Graph Edge"):
+ * e_ij = cosine(x_i, y_j) with x the source node's row of tensor `src_tensor` and y the rows of
+ * tensor `all_tensor` (graphkv_tensor: K or V, with the strides the params give for it).  K/K is
+ * Eq. 1 and what graphkv_propagate computes; V/V and K/V are the value-to-value and key-to-value
+ * variants.  (Query-to-key and query-to-query edges would need the queries of every prefix token,
+ * which a prefill-time cache does not hold.)  A tensor that is not used may be NULL. */
+graphkv_status graphkv_propagate_edges(const graphkv_params *params, const void *K, const void *V,
+                                       int32_t src_tensor, int32_t all_tensor, float *scores,
+                                       int32_t *src_idx_out, void *workspace,
+                                       size_t workspace_bytes, void *stream);
 
 /* Step (IV), "Select Important Tokens": per head the B highest scores (ties: lower index),
  * written to idx_out in ascending position, and the compact cache

@@ -55,6 +55,9 @@ typedef struct {
     int32_t neighbors;   /* m; 0 = adaptive */
     int32_t rounds;      /* T */
     double  decay;       /* lambda */
+    int32_t pool_mode;   /* 0 = max pooling, 1 = mean over kp positions, zeros outside the row */
+    int32_t signal;      /* 0 = decay (Eq. 4-5), 1 = enhanced (1 + lambda e), 2 = evicted (-inf) */
+    int32_t reselect;    /* 1 = sources and neighbourhoods rebuilt before every round */
 } okv_params;
 
 /* ---- adaptive neighbour count: "input length x 1e-3", floored, kept within [1, 32] ---- */
@@ -100,7 +103,7 @@ void okv_topk(const float *x, int32_t n, int32_t k, int32_t skip, int32_t *idx_o
  * Qg [G][W][D], Kh [L][D] (exact input values widened to fp32).
  * a_out (optional) [N] fp64: attention mass before pooling.  s_out [N] fp32: pooled score. */
 void okv_score_unit(const float *Qg, const float *Kh, int32_t G, int32_t W, int32_t D,
-                    int32_t N, int32_t kp, double *a_out, float *s_out)
+                    int32_t N, int32_t kp, int32_t pool_mode, double *a_out, float *s_out)
 {
     const int32_t L = N + W;
     double *a = (double *)calloc((size_t)N, sizeof(double));
@@ -131,8 +134,15 @@ void okv_score_unit(const float *Qg, const float *Kh, int32_t G, int32_t W, int3
         int32_t lo = j - half < 0 ? 0 : j - half;
         int32_t hi = j + half > N - 1 ? N - 1 : j + half;
         double best = a[lo];
-        for (int32_t t = lo + 1; t <= hi; ++t)
-            if (a[t] > best) best = a[t];
+        if (pool_mode == 1) {
+            /* mean pooling as the common SnapKV implementations do it: zeros outside the row,
+             * divided by the kernel size */
+            for (int32_t t = lo + 1; t <= hi; ++t) best += a[t];
+            best /= (double)kp;
+        } else {
+            for (int32_t t = lo + 1; t <= hi; ++t)
+                if (a[t] > best) best = a[t];
+        }
         s_out[j] = (float)best;
     }
     if (a_out) memcpy(a_out, a, (size_t)N * sizeof(double));
@@ -140,10 +150,29 @@ void okv_score_unit(const float *Qg, const float *Kh, int32_t G, int32_t W, int3
     free(l);
 }
 
-/* ---- Eq. 1: edges of one source node to every prefix node ------------------------------ */
-void okv_edges_unit(const float *Kh, int32_t N, int32_t D, int32_t i, double *e_out)
+/* ---- another initial score: KNorm (Experimental Setup, baselines: "applies L2 norm of keys") ----
+ * The cited method keeps the keys of LOWEST L2 norm; the paper gives no formula.  Reading used
+ * here: s_j = 1 / max(||k_j||_2, 1e-12), which ranks like ascending norm and is positive, as the
+ * multiplicative decay of Eq. 5 needs (a negative score would gain rank under a factor in [0,1]).
+ * Kh [L][D]; s_out [N] fp32. */
+void okv_score_knorm_unit(const float *Kh, int32_t N, int32_t D, float *s_out)
 {
-    const float *ki = Kh + (size_t)i * D;
+    for (int32_t j = 0; j < N; ++j) {
+        const float *k = Kh + (size_t)j * D;
+        double n2 = 0.0;
+        for (int32_t d = 0; d < D; ++d) n2 += (double)k[d] * (double)k[d];
+        double n = sqrt(n2);
+        if (n < 1e-12) n = 1e-12;
+        s_out[j] = (float)(1.0 / n);
+    }
+}
+
+/* ---- Eq. 1: edges of one source node to every prefix node ------------------------------
+ * e_ij = cosine(S[i], A[j]): S = A = the keys for Eq. 1; keys and values, or values and values,
+ * for the other edge kinds of the Discussion. */
+void okv_edges2_unit(const float *Sh, const float *Kh, int32_t N, int32_t D, int32_t i, double *e_out)
+{
+    const float *ki = Sh + (size_t)i * D;
     double ni = 0.0;
     for (int32_t d = 0; d < D; ++d) ni += (double)ki[d] * (double)ki[d];
     ni = sqrt(ni);
@@ -164,14 +193,19 @@ void okv_edges_unit(const float *Kh, int32_t N, int32_t D, int32_t i, double *e_
     }
 }
 
+void okv_edges_unit(const float *Kh, int32_t N, int32_t D, int32_t i, double *e_out)
+{
+    okv_edges2_unit(Kh, Kh, N, D, i, e_out);
+}
+
 /* ---- steps (II)+(III): sparse graph + T rounds of decay on one KV head ------------------
  * s [N] fp32, updated in place.  forced_src (optional, [K_src]) replaces the top-K_src pick;
  * forced_nbr (optional, [K_src][m]) replaces the top-m pick of each source.
  * Outputs (each optional): src_out [K_src], nbr_out [K_src][m], nbr_e_out [K_src][m] fp64. */
-void okv_propagate_unit(const float *Kh, int32_t N, int32_t D, float *s, int32_t K_src,
-                        int32_t m, int32_t T, double lambda, const int32_t *forced_src,
-                        const int32_t *forced_nbr, int32_t *src_out, int32_t *nbr_out,
-                        double *nbr_e_out)
+void okv_propagate2_unit(const float *Sh, const float *Kh, int32_t N, int32_t D, float *s, int32_t K_src,
+                         int32_t m, int32_t T, double lambda, int32_t signal, const int32_t *forced_src,
+                         const int32_t *forced_nbr, int32_t *src_out, int32_t *nbr_out,
+                         double *nbr_e_out)
 {
     if (K_src <= 0 || m <= 0) return;
     int32_t *src = (int32_t *)malloc((size_t)K_src * sizeof(int32_t));
@@ -187,7 +221,7 @@ void okv_propagate_unit(const float *Kh, int32_t N, int32_t D, float *s, int32_t
     /* Eq. 1 + Eq. 3: edges of each source, and its top-m neighbourhood (j != i) */
     for (int32_t a = 0; a < K_src; ++a) {
         const int32_t i = src[a];
-        okv_edges_unit(Kh, N, D, i, e);
+        okv_edges2_unit(Sh, Kh, N, D, i, e);
         if (forced_nbr) memcpy(nbr + (size_t)a * m, forced_nbr + (size_t)a * m,
                                (size_t)m * sizeof(int32_t));
         else {
@@ -206,7 +240,9 @@ void okv_propagate_unit(const float *Kh, int32_t N, int32_t D, float *s, int32_t
                 const int32_t j = nbr[(size_t)a * m + u];
                 double eij = nbr_e[(size_t)a * m + u];
                 if (eij < 0.0) eij = 0.0;
-                cur[j] = cur[j] * (1.0 - lambda * eij);
+                if (signal == 2) cur[j] = -INFINITY;                        /* evicted */
+                else if (signal == 1) cur[j] = cur[j] * (1.0 + lambda * eij); /* enhanced */
+                else cur[j] = cur[j] * (1.0 - lambda * eij);                /* decay, Eq. 5 */
             }
         }
     }
@@ -216,6 +252,26 @@ void okv_propagate_unit(const float *Kh, int32_t N, int32_t D, float *s, int32_t
     if (nbr_out) memcpy(nbr_out, nbr, (size_t)K_src * m * sizeof(int32_t));
     if (nbr_e_out) memcpy(nbr_e_out, nbr_e, (size_t)K_src * m * sizeof(double));
     free(cur); free(e32); free(e); free(nbr_e); free(nbr); free(src);
+}
+
+void okv_propagate_unit(const float *Kh, int32_t N, int32_t D, float *s, int32_t K_src,
+                        int32_t m, int32_t T, double lambda, const int32_t *forced_src,
+                        const int32_t *forced_nbr, int32_t *src_out, int32_t *nbr_out,
+                        double *nbr_e_out)
+{
+    okv_propagate2_unit(Kh, Kh, N, D, s, K_src, m, T, lambda, 0, forced_src, forced_nbr, src_out,
+                        nbr_out, nbr_e_out);
+}
+
+/* The other reading of "dynamically updated ... one or multiple times": every round re-picks the
+ * sources from the scores the round before left (as fp32, the precision the score arrays have)
+ * and rebuilds their neighbourhoods: T passes of Algorithm 1 + one round of Algorithm 2. */
+void okv_propagate_reselect_unit(const float *Sh, const float *Kh, int32_t N, int32_t D, float *s,
+                                 int32_t K_src, int32_t m, int32_t T, double lambda, int32_t signal,
+                                 int32_t *src_out)
+{
+    for (int32_t t = 0; t < T; ++t)
+        okv_propagate2_unit(Sh, Kh, N, D, s, K_src, m, 1, lambda, signal, NULL, NULL, src_out, NULL, NULL);
 }
 
 /* ---- step (IV): keep the B highest scores, ascending position --------------------------- */
@@ -262,7 +318,7 @@ void okv_score(const okv_params *p, const float *Qw, const float *K, float *scor
         const int32_t b = u / p->n_kv_heads, h = u % p->n_kv_heads;
         const float *Qg = Qw + (((size_t)b * p->n_q_heads + (size_t)h * G) * W) * D;
         const float *Kh = K + ((size_t)u * L) * D;
-        okv_score_unit(Qg, Kh, G, W, D, N, p->pool_kernel, NULL, scores + (size_t)u * N);
+        okv_score_unit(Qg, Kh, G, W, D, N, p->pool_kernel, p->pool_mode, NULL, scores + (size_t)u * N);
     }
 }
 
@@ -281,9 +337,14 @@ void okv_propagate(const okv_params *p, const float *K, float *scores, int32_t *
     }
 #pragma omp parallel for schedule(dynamic, 1)
     for (int32_t u = 0; u < units; ++u) {
-        okv_propagate_unit(K + ((size_t)u * L) * D, N, D, scores + (size_t)u * N,
-                           p->topk_nodes, m, p->rounds, p->decay, NULL, NULL,
-                           src_out ? src_out + (size_t)u * p->topk_nodes : NULL, NULL, NULL);
+        const float *Kh = K + ((size_t)u * L) * D;
+        int32_t *so = src_out ? src_out + (size_t)u * p->topk_nodes : NULL;
+        if (p->reselect)
+            okv_propagate_reselect_unit(Kh, Kh, N, D, scores + (size_t)u * N, p->topk_nodes, m, p->rounds,
+                                        p->decay, p->signal, so);
+        else
+            okv_propagate2_unit(Kh, Kh, N, D, scores + (size_t)u * N, p->topk_nodes, m, p->rounds,
+                                p->decay, p->signal, NULL, NULL, so, NULL, NULL);
     }
 }
 

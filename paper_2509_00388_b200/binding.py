@@ -19,12 +19,16 @@ LIB_PATH = os.environ.get("GRAPHKV_LIB") or os.path.join(HERE, "libgraphkv.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BUILTIN_SCRATCH = range(7)
 BUILTIN_SCRATCH_BYTES = 16 << 20
 BF16, F32 = 0, 1
+POOL_MAX, POOL_AVG = 0, 1
+SIGNAL_DECAY, SIGNAL_ENHANCE, SIGNAL_EVICT = 0, 1, 2
+TENSOR_K, TENSOR_V = 0, 1
 
 EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_score",
            "graphkv_propagate", "graphkv_select_gather", "graphkv_compress",
            "graphkv_read_status", "graphkv_status_string", "graphkv_launch_count",
            "graphkv_trace_enable", "graphkv_trace_read", "graphkv_builtin_scratch_needed",
-           "graphkv_score_noalloc", "graphkv_read_status_noalloc", "graphkv_read_neighbors", "graphkv_phase_timing_read")
+           "graphkv_score_noalloc", "graphkv_read_status_noalloc", "graphkv_read_neighbors", "graphkv_phase_timing_read", "graphkv_score_knorm",
+           "graphkv_propagate_edges")
 
 
 class GraphKVError(RuntimeError):
@@ -40,7 +44,7 @@ class Params(C.Structure):
                 ("topk_nodes", C.c_int32), ("neighbors", C.c_int32), ("rounds", C.c_int32),
                 ("decay", C.c_float), ("dtype", C.c_int32),
                 ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
-                ("v_stride", C.c_int64 * 3)]
+                ("v_stride", C.c_int64 * 3), ("signal", C.c_int32), ("reselect", C.c_int32)]
 
 
 class TraceRecord(C.Structure):
@@ -75,6 +79,10 @@ def lib() -> C.CDLL:
         L.graphkv_compress.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.graphkv_read_status.restype = C.c_int
         L.graphkv_read_status.argtypes = [vp, vp]
+        L.graphkv_score_knorm.restype = C.c_int
+        L.graphkv_score_knorm.argtypes = [P, vp, vp, vp]
+        L.graphkv_propagate_edges.restype = C.c_int
+        L.graphkv_propagate_edges.argtypes = [P, vp, vp, C.c_int32, C.c_int32, vp, vp, vp, sz, vp]
         L.graphkv_read_neighbors.restype = C.c_int
         L.graphkv_read_neighbors.argtypes = [P, vp, sz, vp, vp, vp]
         L.graphkv_phase_timing_read.restype = C.c_int32
@@ -123,13 +131,15 @@ def _strides3(t: Optional[torch.Tensor]):
 def make_params(K: torch.Tensor, *, window: int, n_q_heads: Optional[int] = None,
                 Qw: Optional[torch.Tensor] = None, V: Optional[torch.Tensor] = None,
                 budget: int = 1, pool_kernel: int = 1, topk_nodes: int = 0, neighbors: int = 0,
-                rounds: int = 0, decay: float = 1.0) -> Params:
+                rounds: int = 0, decay: float = 1.0, pool_mode: int = 0, signal: int = 0,
+                reselect: int = 0) -> Params:
     b, hkv, ell, d = K.shape
     hq = Qw.shape[1] if Qw is not None else (n_q_heads or hkv)
     p = Params()
     p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = b, hq, hkv, d
     p.seq_len, p.window, p.budget = ell, window, budget
-    p.pool_kernel, p.pool_mode = pool_kernel, 0
+    p.pool_kernel, p.pool_mode = pool_kernel, pool_mode
+    p.signal, p.reselect = signal, reselect
     p.topk_nodes, p.neighbors, p.rounds, p.decay = topk_nodes, neighbors, rounds, decay
     p.dtype = _dtype_code(K)
     p.q_stride = _strides3(Qw)
@@ -146,7 +156,8 @@ def alloc_workspace(p: Params, device) -> torch.Tensor:
     n = workspace_bytes(p)
     if n == 0:
         raise GraphKVError(ERR_INVALID_ARG, "graphkv_workspace_bytes")
-    return torch.empty(n, dtype=torch.uint8, device=device)
+    # zero-filled: the status word at its head is only cleared by the scoring calls
+    return torch.zeros(n, dtype=torch.uint8, device=device)
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -189,6 +200,19 @@ def graphkv_propagate(p: Params, K: torch.Tensor, scores: torch.Tensor,
     _check(lib().graphkv_propagate(C.byref(p), _ptr(K), _ptr(scores), _ptr(src_idx_out),
                                    _ptr(ws), ws.numel(), _stream(K.device)),
            "graphkv_propagate")
+
+
+def graphkv_score_knorm(p: Params, K: torch.Tensor, scores: torch.Tensor) -> None:
+    _check(lib().graphkv_score_knorm(C.byref(p), _ptr(K), _ptr(scores), _stream(K.device)),
+           "graphkv_score_knorm")
+
+
+def graphkv_propagate_edges(p: Params, K: Optional[torch.Tensor], V: Optional[torch.Tensor],
+                            src_tensor: int, all_tensor: int, scores: torch.Tensor,
+                            src_idx_out: Optional[torch.Tensor], ws: torch.Tensor) -> None:
+    _check(lib().graphkv_propagate_edges(C.byref(p), _ptr(K), _ptr(V), src_tensor, all_tensor,
+                                         _ptr(scores), _ptr(src_idx_out), _ptr(ws), ws.numel(),
+                                         _stream(scores.device)), "graphkv_propagate_edges")
 
 
 def graphkv_select_gather(p: Params, scores: torch.Tensor, K: Optional[torch.Tensor],

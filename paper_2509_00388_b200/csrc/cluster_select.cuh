@@ -594,6 +594,7 @@ struct PushLists {
     int slot0;
     float lambda;
     int T;
+    int signal;
 };
 
 __device__ void merge_neighbours(cg::cluster_group &cl, const Cand *cand, const uint32_t *hist,
@@ -674,9 +675,7 @@ __device__ void merge_neighbours(cg::cluster_group &cl, const Cand *cand, const 
         if (rank < m) {
             nbr_idx[rank] = me.j;
             nbr_e[rank] = me.e;
-            const float f = 1.0f - push.lambda * fmaxf(me.e, 0.f);
-            float pw = f;
-            for (int t = 1; t < push.T; ++t) pw *= f;
+            const float pw = signal_factor(me.e, push.lambda, push.T, push.signal);
             for (int p = 0; p < push.R; ++p) {
                 (push.C > 1 ? cl.map_shared_rank(push.nb_j, p) : push.nb_j)[push.slot0 + rank] = me.j;
                 (push.C > 1 ? cl.map_shared_rank(push.nb_f, p) : push.nb_f)[push.slot0 + rank] = pw;
@@ -877,7 +876,8 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
         for (int i = rank * kThreads + tid; i < a.zero_words; i += C * kThreads)
             a.zero[(long long)unit * a.zero_words + i] = 0u;
     // this thread's two counts of the mass histogram, on their way while the row is pooled
-    const bool bounded = a.mass_hist && a.k > 0 && a.k <= kThreads;
+    // (the bound from the mass histogram needs pooling that only raises values: max pooling)
+    const bool bounded = a.mass_hist && a.k > 0 && a.k <= kThreads && !a.d.pool_avg;
     uint32_t hc0 = 0, hc1 = 0;
     if (bounded) {
         const uint32_t *mh = a.mass_hist + (long long)unit * kBins;
@@ -887,7 +887,8 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
     if (a.a) {
         const float *row_a = a.a + (long long)unit * N;
         const int half = a.halo;
-        if (n_local > 0) load_chunk(row_a, base, -half, n_local + half, N, vals, -INFINITY);
+        const bool avg = a.d.pool_avg != 0;
+        if (n_local > 0) load_chunk(row_a, base, -half, n_local + half, N, vals, avg ? 0.f : -INFINITY);
         __syncthreads();
         float pooled[kPer];
 #pragma unroll
@@ -895,7 +896,13 @@ __global__ void __launch_bounds__(kThreads, 1) pool_select_kernel(PoolSelectArgs
             const int i = q * kThreads + tid;
             if (i < n_local) {
                 float best = vals[i - half];
-                for (int t = 1 - half; t <= half; ++t) best = fmaxf(best, vals[i + t]);
+                if (avg) {
+                    // ascending positions, zeros outside the row, divided by the kernel size
+                    for (int t = 1 - half; t <= half; ++t) best += vals[i + t];
+                    best /= (float)(2 * half + 1);
+                } else {
+                    for (int t = 1 - half; t <= half; ++t) best = fmaxf(best, vals[i + t]);
+                }
                 pooled[q] = best;
             }
         }
@@ -1039,12 +1046,13 @@ __device__ void store_chunk(float *row, const float *vals, int n)
 }
 
 // Eq. 5 on the chunk in shared memory: the unit's lists are in s.nb_j / s.nb_f as (position,
-// factor over all rounds).  A position that only one listed edge points to (counted per slot of a
+// factor over all rounds); with the evicted signal every listed position becomes -inf instead.  A position that only one listed edge points to (counted per slot of a
 // small table, so a slot shared with another position counts as contested) takes its factor at
 // once; the contested ones are applied by one warp, source after source (a source's neighbours are
 // distinct), so that overlapping neighbourhoods multiply in a fixed order.  Uses s.fine as
 // scratch.  Ends with the CTA synchronised.
-__device__ void apply_lists(const Smem &s, float *vals, int base, int n_local, int K_src, int m)
+__device__ void apply_lists(const Smem &s, float *vals, int base, int n_local, int K_src, int m,
+                            bool evict)
 {
     const int tid = threadIdx.x;
     const int pairs = K_src * m;                           // <= kStage, so K_src <= kStage
@@ -1060,7 +1068,9 @@ __device__ void apply_lists(const Smem &s, float *vals, int base, int n_local, i
     for (int p = tid; p < pairs; p += kThreads) {
         const int j = s.nb_j[p] - base;
         if (j >= 0 && j < n_local) {
-            if (cnt[j & 4095] == 1u) {
+            if (evict) {
+                vals[j] = -INFINITY;                       // the evicted signal: no order to keep
+            } else if (cnt[j & 4095] == 1u) {
                 vals[j] *= s.nb_f[p];
             } else {
                 const int q = p / m;
@@ -1164,7 +1174,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
                 const int M = spare_first ? C - 1 : C, mr = spare_first ? rank - 1 : rank;
                 for (int src = grp * M + mr; mr >= 0 && src < d.K_src; src += kMergeWarps * M) {
                     const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
-                    const PushLists push{C, R, s.nb_j, s.nb_f, src * d.m, d.lambda, d.T};
+                    const PushLists push{C, R, s.nb_j, s.nb_f, src * d.m, d.lambda, d.T, d.signal};
                     merge_neighbours(cl, a.cand + slot * kCandCap,
                                      a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
                                      a.cand_chunks, d.m, surv, ns_sh, 1 + grp, wg, ni + src * d.m,
@@ -1175,25 +1185,19 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
                 pc.mark();
             } else if (holds) {
                 for (int i = tid; i < pairs; i += kThreads) {
-                    const float f = 1.0f - d.lambda * fmaxf(__ldcg(ne + i), 0.f);
-                    float pw = f;
-                    for (int t = 1; t < d.T; ++t) pw *= f;
                     s.nb_j[i] = __ldcg(ni + i);
-                    s.nb_f[i] = pw;
+                    s.nb_f[i] = signal_factor(__ldcg(ne + i), d.lambda, d.T, d.signal);
                 }
                 __syncthreads();
             }
-            if (holds) apply_lists(s, vals, base, n_local, d.K_src, d.m);
+            if (holds) apply_lists(s, vals, base, n_local, d.K_src, d.m, d.signal == GRAPHKV_SIGNAL_EVICT);
         } else if (holds) {
             for (int src = 0; src < d.K_src; ++src) {
                 for (int u = tid; u < d.m; u += kThreads) {
                     const int j = ni[src * d.m + u] - base;
-                    if (j >= 0 && j < n_local) {
-                        const float f = 1.0f - d.lambda * fmaxf(ne[src * d.m + u], 0.f);
-                        float pw = f;
-                        for (int t = 1; t < d.T; ++t) pw *= f;
-                        vals[j] *= pw;
-                    }
+                    if (j >= 0 && j < n_local)
+                        vals[j] = d.signal == GRAPHKV_SIGNAL_EVICT
+                                      ? -INFINITY : vals[j] * signal_factor(ne[src * d.m + u], d.lambda, d.T, d.signal);
                 }
                 __syncthreads();
             }

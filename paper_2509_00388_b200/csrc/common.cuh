@@ -22,6 +22,9 @@ struct Dims {
     float lambda;
     int units;                 // batch * hkv independent (sequence, KV head) problems
     int bf16;                  // inputs are bf16 (else fp32)
+    int pool_avg;              // mean pooling (zeros outside the row) instead of max pooling
+    int signal;                // graphkv_signal
+    int reselect;              // sources re-picked every round
     long long qs[3], ks[3], vs[3];
 };
 
@@ -127,6 +130,18 @@ struct PhaseClock {
     __device__ __forceinline__ void flush(int) {}
 };
 #endif
+
+// What a listed edge of cosine e does to its neighbour's score over T rounds of a fixed graph, as
+// a factor: (1 - lambda*max(e,0))^T for the decay signal, (1 + lambda*max(e,0))^T for the enhanced
+// one.  (The evicted signal is no factor: the score becomes -inf.)
+__device__ __forceinline__ float signal_factor(float e, float lambda, int T, int signal)
+{
+    const float x = lambda * fmaxf(e, 0.f);
+    const float f = signal == GRAPHKV_SIGNAL_ENHANCE ? 1.0f + x : 1.0f - x;
+    float pw = f;
+    for (int t = 1; t < T; ++t) pw *= f;
+    return pw;
+}
 
 __device__ __forceinline__ float warp_sum(float v)
 {

@@ -60,7 +60,9 @@ graphkv_status resolve(const graphkv_params *p, Dims *d)
     if (p->rounds < 0) return GRAPHKV_ERR_INVALID_ARG;
     if (!(p->decay >= 0.0f && p->decay <= 1.0f)) return GRAPHKV_ERR_INVALID_ARG;
     if (p->dtype != GRAPHKV_BF16 && p->dtype != GRAPHKV_F32) return GRAPHKV_ERR_INVALID_ARG;
-    if (p->pool_mode != GRAPHKV_POOL_MAX) return GRAPHKV_ERR_UNSUPPORTED;
+    if (p->pool_mode != GRAPHKV_POOL_MAX && p->pool_mode != GRAPHKV_POOL_AVG) return GRAPHKV_ERR_INVALID_ARG;
+    if (p->signal < GRAPHKV_SIGNAL_DECAY || p->signal > GRAPHKV_SIGNAL_EVICT) return GRAPHKV_ERR_INVALID_ARG;
+    if (p->reselect != 0 && p->reselect != 1) return GRAPHKV_ERR_INVALID_ARG;
     if (p->head_dim != kHeadDim) return GRAPHKV_ERR_UNSUPPORTED;
     const int G = p->n_q_heads / p->n_kv_heads;
     if ((long long)G * p->window > kMaxRows) return GRAPHKV_ERR_UNSUPPORTED;
@@ -80,6 +82,9 @@ graphkv_status resolve(const graphkv_params *p, Dims *d)
     d->m = graphkv_resolve_neighbors(N, p->neighbors);
     d->T = p->rounds; d->lambda = p->decay; d->units = p->batch * p->n_kv_heads;
     d->bf16 = p->dtype == GRAPHKV_BF16 ? 1 : 0;
+    d->pool_avg = p->pool_mode == GRAPHKV_POOL_AVG ? 1 : 0;
+    d->signal = p->signal;
+    d->reselect = p->reselect;
     for (int i = 0; i < 3; ++i) {
         d->qs[i] = p->q_stride[i]; d->ks[i] = p->k_stride[i]; d->vs[i] = p->v_stride[i];
     }
@@ -396,13 +401,14 @@ EncodeTiledFn encode_tiled_fn()
 
 // Tensor map over K [batch][hkv][rows][128] bf16 with the caller's strides; boxes of 128 rows x 64
 // columns, 128-byte swizzle, zero fill past the last row.
-bool make_k_tensormap(CUtensorMap *tm, const void *K, const Dims &d, int rows)
+bool make_k_tensormap(CUtensorMap *tm, const void *K, const Dims &d, int rows, const long long *ks = nullptr)
 {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
-    const cuuint64_t row_b = (cuuint64_t)d.ks[2] * 2;
+    if (!ks) ks = d.ks;
+    const cuuint64_t row_b = (cuuint64_t)ks[2] * 2;
     cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows, (cuuint64_t)d.hkv, (cuuint64_t)d.batch};
-    cuuint64_t head_b = (cuuint64_t)d.ks[1] * 2, batch_b = (cuuint64_t)d.ks[0] * 2;
+    cuuint64_t head_b = (cuuint64_t)ks[1] * 2, batch_b = (cuuint64_t)ks[0] * 2;
     if (d.hkv == 1 || head_b == 0) head_b = row_b * (cuuint64_t)rows;
     if (d.batch == 1 || batch_b == 0) batch_b = head_b * (cuuint64_t)d.hkv;
     cuuint64_t strides[3] = {row_b, head_b, batch_b};
@@ -537,7 +543,7 @@ graphkv_status run_pool_sources(const Dims &d, const float *a, float *s, int k, 
         return GRAPHKV_ERR_CUDA;
     if (a)
         GKV_LAUNCH("pool_max", st,
-                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a, s)));
+                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, d.pool_avg, a, s)));
     if (k > 0) {
         SelectArgs sa{s, d.N, d.N, k, nullptr, src, nullptr};
         GKV_LAUNCH("select_sources", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
@@ -550,14 +556,22 @@ inline bool graph_active(const Dims &d) { return d.K_src > 0 && d.T > 0 && d.m >
 
 // Edges of the sources (Eq. 1) and their top-m neighbourhoods (Eq. 3) -> neighbour lists in the
 // workspace.  `src` holds the sources in ascending position.
+// The tensors an edge compares: the sources' vectors come from S, the swept vectors from A.
+template <typename T> struct EdgeOperands {
+    const T *S;
+    const long long *ss;
+    const T *A;
+    const long long *as;
+};
+
 template <typename T>
-graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *src, void *ws,
+graphkv_status run_graph(const Dims &d, const Layout &l, const EdgeOperands<T> &eo, const int *src, void *ws,
                          cudaStream_t st)
 {
     const SimPlan sp = sim_plan(d, sizeof(T) == 2);
     if (sp.ok) {
         CUtensorMap tmK;
-        if (!make_k_tensormap(&tmK, K, d, d.L)) return GRAPHKV_ERR_CUDA;
+        if (!make_k_tensormap(&tmK, eo.A, d, d.L, eo.as)) return GRAPHKV_ERR_CUDA;
         static std::mutex mu;
         static signed char state[64] = {};
         if (!once_per_device(mu, state, [] {
@@ -569,7 +583,7 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *
         const int group = units_per_group(d);
         for (int u0 = 0; u0 < d.units; u0 += group) {
             const int nu = std::min(group, d.units - u0);
-            tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(K), src, at<Cand>(ws, l.cand),
+            tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(eo.S), {eo.ss[0], eo.ss[1], eo.ss[2]}, src, at<Cand>(ws, l.cand),
                              at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
                              sp.n_tiles, sp.stages, 0, wait_cycles()};
             sa.wait_prior = next_launch_is_dependent();
@@ -591,7 +605,8 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const T *K, const int *
     float *sims = at<float>(ws, l.sims);
     GKV_LAUNCH("similarity_simt", st,
                (similarity_simt<T><<<dim3(ceil_div(d.N, kSimChunk), d.units), kSimThreads, 0, st>>>(
-                   d, K, src, sims)));
+                   d, eo.S, Strides3{{eo.ss[0], eo.ss[1], eo.ss[2]}}, eo.A, Strides3{{eo.as[0], eo.as[1], eo.as[2]}},
+                   src, sims)));
     SelectArgs na{sims, d.N, d.N, d.m, src, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e)};
     GKV_LAUNCH("select_neighbors", st,
                (topk_select_kernel<<<d.units * d.K_src, kSelectThreads, 0, st>>>(na)));
@@ -637,7 +652,7 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const 
     }
     if (a)
         GKV_LAUNCH("pool_max", st,
-                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, a, s)));
+                   (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, d.pool_avg, a, s)));
     if (has_graph)
         GKV_LAUNCH("decay_rounds", st,
                    (decay_rounds_kernel<<<d.units, 256, 0, st>>>(d, at<int>(ws, l.nbr_idx),
@@ -678,20 +693,39 @@ graphkv_status do_score(const Dims &d, const Layout &l, const T *Q, const T *K, 
     return run_pool_sources(d, a, scores, 0, nullptr, nullptr, nullptr, 0, st);
 }
 
+// One pass of steps (II)+(III) from the scores as they stand: sources, edges, neighbourhoods,
+// d.T rounds over that graph.
 template <typename T>
-graphkv_status do_propagate(const Dims &d, const Layout &l, const T *K, float *scores, int *src_out,
-                            void *ws, cudaStream_t st)
+graphkv_status propagate_once(const Dims &d, const Layout &l, const EdgeOperands<T> &eo, float *scores,
+                              int *src, void *ws, cudaStream_t st)
 {
-    if (d.K_src == 0) return GRAPHKV_OK;
-    int *src = src_out ? src_out : at<int>(ws, l.src);
     const bool tc_graph = graph_active(d) && sim_plan(d, sizeof(T) == 2).ok;
     graphkv_status rc = run_pool_sources(d, nullptr, scores, d.K_src, src, nullptr,
                                          tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr,
                                          d.K_src * kCandBins, st);
     if (rc != GRAPHKV_OK || !graph_active(d)) return rc;
-    if ((rc = run_graph(d, l, K, src, ws, st)) != GRAPHKV_OK) return rc;
+    if ((rc = run_graph(d, l, eo, src, ws, st)) != GRAPHKV_OK) return rc;
     return run_finish(d, l, (int)sizeof(T), nullptr, scores, true, sim_plan(d, sizeof(T) == 2).ok, false,
                       nullptr, nullptr, nullptr, nullptr, nullptr, ws, st);
+}
+
+// Steps (II)+(III).  With d.reselect every round is a pass of its own: the sources are re-picked
+// from the scores the round before left and their neighbourhoods rebuilt (src_out then holds the
+// sources of the last round).
+template <typename T>
+graphkv_status do_propagate(const Dims &d, const Layout &l, const EdgeOperands<T> &eo, float *scores,
+                            int *src_out, void *ws, cudaStream_t st)
+{
+    if (d.K_src == 0) return GRAPHKV_OK;
+    int *src = src_out ? src_out : at<int>(ws, l.src);
+    if (!d.reselect || d.T <= 1) return propagate_once(d, l, eo, scores, src, ws, st);
+    Dims one = d;
+    one.T = 1;
+    for (int t = 0; t < d.T; ++t) {
+        const graphkv_status rc = propagate_once(one, l, eo, scores, src, ws, st);
+        if (rc != GRAPHKV_OK) return rc;
+    }
+    return GRAPHKV_OK;
 }
 
 template <typename T>
@@ -708,8 +742,10 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
     // The tensor-core emit sweep can pick the sources at its tail and the finishing kernel can pool,
     // which saves the pooling kernel's launch; measured on B200 the serial tail of the unit's last
     // emit CTA (about 12 us at 32K keys) costs more than that kernel (10 us), so it is off by default.
-    const bool tail_src = tc_mass(Q) && tc_graph && d.K_src <= tc::kSrcMaxK && env_int("GRAPHKV_TAIL_SOURCES", 0);
-    const bool finish_pools = d.kp > 1 && (tail_src || !graph) && finish_plan(d, halo).ok && cluster_plan(d).ok;
+    const bool tail_src = tc_mass(Q) && tc_graph && d.K_src <= tc::kSrcMaxK && !d.pool_avg &&
+                          env_int("GRAPHKV_TAIL_SOURCES", 0);
+    const bool finish_pools = d.kp > 1 && !d.pool_avg && (tail_src || !graph) && finish_plan(d, halo).ok &&
+                              cluster_plan(d).ok;
     graphkv_status rc;
     if (tail_src || !graph) {
         const EmitExtras ex{tail_src ? d.K_src : 0, src, tail_src ? at<uint32_t>(ws, l.cand_hist) : nullptr,
@@ -726,9 +762,58 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
                               tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr, d.K_src * kCandBins, st);
         if (rc != GRAPHKV_OK) return rc;
     }
-    if (graph && (rc = run_graph(d, l, K, src, ws, st)) != GRAPHKV_OK) return rc;
+    const EdgeOperands<T> eo{K, d.ks, K, d.ks};
+    if (graph && d.reselect && d.T > 1) {
+        // every round its own pass: the first one rides on the sources picked above, the rounds
+        // after it start from the scores in `s`; the last pass also selects and gathers
+        Dims one = d;
+        one.T = 1;
+        if ((rc = run_graph(one, l, eo, src, ws, st)) != GRAPHKV_OK) return rc;
+        if ((rc = run_finish(one, l, (int)sizeof(T), finish_pools ? a : nullptr, s, true, tc_graph, false,
+                             nullptr, nullptr, nullptr, nullptr, nullptr, ws, st)) != GRAPHKV_OK)
+            return rc;
+        for (int t = 1; t < d.T; ++t)
+            if ((rc = propagate_once(one, l, eo, s, src, ws, st)) != GRAPHKV_OK) return rc;
+        return run_finish(one, l, (int)sizeof(T), nullptr, s, false, false, true, K, V, K_out, V_out, idx_out,
+                          ws, st);
+    }
+    if (graph && (rc = run_graph(d, l, eo, src, ws, st)) != GRAPHKV_OK) return rc;
     return run_finish(d, l, (int)sizeof(T), finish_pools ? a : nullptr, s, graph, tc_graph, true, K, V,
                       K_out, V_out, idx_out, ws, st);
+}
+
+// ---- KNorm initial score ---------------------------------------------------------------------
+// s_j = 1 / max(||k_j||, eps) for the prefix keys: 16 threads share a key row (16 bytes each of a
+// bf16 row, 32 of an fp32 row), four rows in flight per thread.  grid-stride over units * N rows.
+template <typename T>
+__global__ void __launch_bounds__(256) knorm_score_kernel(Dims d, const T *__restrict__ K, float *__restrict__ scores)
+{
+    const int sub = threadIdx.x & 15;
+    const long long rows = (long long)d.units * d.N;
+    const long long stride = ((long long)gridDim.x * blockDim.x) >> 4;
+    for (long long r0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 4; r0 < rows; r0 += 4 * stride) {
+        float n2[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long r = r0 + u * stride;
+            n2[u] = 0.f;
+            if (r < rows) {
+                const int unit = (int)(r / d.N), j = (int)(r % d.N);
+                const T *row = K + (unit / d.hkv) * d.ks[0] + (long long)(unit % d.hkv) * d.ks[1] + (long long)j * d.ks[2];
+                float v[8];
+                load8(row + sub * 8, v);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) n2[u] = fmaf(v[e], v[e], n2[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) n2[u] += __shfl_xor_sync(0xffffffffu, n2[u], o);
+            const long long r = r0 + u * stride;
+            if (sub == 0 && r < rows) scores[r] = 1.0f / fmaxf(sqrtf(n2[u]), kNormEps);
+        }
+    }
 }
 
 // ---- built-in scratch for graphkv_score_noalloc ---------------------------------------------------
@@ -825,22 +910,58 @@ graphkv_status graphkv_read_status_noalloc(void *stream)
     return graphkv_read_status(ws, stream);
 }
 
-graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, float *scores,
-                                 int32_t *src_idx_out, void *workspace, size_t workspace_bytes,
-                                 void *stream)
+graphkv_status graphkv_propagate_edges(const graphkv_params *params, const void *K, const void *V,
+                                       int32_t src_tensor, int32_t all_tensor, float *scores,
+                                       int32_t *src_idx_out, void *workspace, size_t workspace_bytes,
+                                       void *stream)
 {
     Dims d;
     graphkv_status rc = resolve(params, &d);
     if (rc != GRAPHKV_OK) return rc;
     t_launches_in_call = 0;
-    if (!K || !scores || !aligned16(K)) return GRAPHKV_ERR_INVALID_ARG;
+    if ((src_tensor != GRAPHKV_TENSOR_K && src_tensor != GRAPHKV_TENSOR_V) ||
+        (all_tensor != GRAPHKV_TENSOR_K && all_tensor != GRAPHKV_TENSOR_V))
+        return GRAPHKV_ERR_INVALID_ARG;
+    const void *S = src_tensor == GRAPHKV_TENSOR_K ? K : V, *A = all_tensor == GRAPHKV_TENSOR_K ? K : V;
+    const long long *ss = src_tensor == GRAPHKV_TENSOR_K ? d.ks : d.vs;
+    const long long *as = all_tensor == GRAPHKV_TENSOR_K ? d.ks : d.vs;
+    if (!S || !A || !scores || !aligned16(S) || !aligned16(A)) return GRAPHKV_ERR_INVALID_ARG;
     const Layout l = layout_of(d);
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (params->dtype == GRAPHKV_BF16) {
+        const EdgeOperands<__nv_bfloat16> eo{static_cast<const __nv_bfloat16 *>(S), ss,
+                                             static_cast<const __nv_bfloat16 *>(A), as};
+        return do_propagate(d, l, eo, scores, src_idx_out, workspace, st);
+    }
+    const EdgeOperands<float> eo{static_cast<const float *>(S), ss, static_cast<const float *>(A), as};
+    return do_propagate(d, l, eo, scores, src_idx_out, workspace, st);
+}
+
+graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, float *scores,
+                                 int32_t *src_idx_out, void *workspace, size_t workspace_bytes,
+                                 void *stream)
+{
+    return graphkv_propagate_edges(params, K, nullptr, GRAPHKV_TENSOR_K, GRAPHKV_TENSOR_K, scores,
+                                   src_idx_out, workspace, workspace_bytes, stream);
+}
+
+graphkv_status graphkv_score_knorm(const graphkv_params *params, const void *K, float *scores, void *stream)
+{
+    Dims d;
+    graphkv_status rc = resolve(params, &d);
+    if (rc != GRAPHKV_OK) return rc;
+    if (!K || !scores || !aligned16(K)) return GRAPHKV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long rows = (long long)d.units * d.N;
+    const int blocks = (int)std::min<long long>((rows * 16 + 255) / 256, (long long)sm_count() * 16);
     if (params->dtype == GRAPHKV_BF16)
-        return do_propagate(d, l, static_cast<const __nv_bfloat16 *>(K), scores, src_idx_out,
-                            workspace, st);
-    return do_propagate(d, l, static_cast<const float *>(K), scores, src_idx_out, workspace, st);
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
+                                          d, static_cast<const __nv_bfloat16 *>(K), scores)));
+    else
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<float><<<blocks, 256, 0, st>>>(
+                                          d, static_cast<const float *>(K), scores)));
+    return launch_status();
 }
 
 graphkv_status graphkv_select_gather(const graphkv_params *params, const float *scores,

@@ -14,14 +14,22 @@ constexpr int kMaxSrcSmem = 64;    // source rows staged per pass over the key r
 // for all sources a of the head and every prefix key j.  Entry j = src[a] is written too; the
 // neighbour selection excludes it by index.
 // grid (ceil(N / kSimChunk), units), block kSimThreads.  sims [units][K_src][N].
+// The sources' vectors come from tensor S (strides ss), the swept vectors from tensor K (strides
+// ks): the same tensor for Eq. 1, keys and values for the other edge kinds.
+struct Strides3 {
+    long long v[3];
+};
+
 template <typename T>
-__global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *__restrict__ K,
+__global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *__restrict__ S, Strides3 ss,
+                                                             const T *__restrict__ K, Strides3 ks,
                                                              const int *__restrict__ src,
                                                              float *__restrict__ sims)
 {
     __shared__ __align__(16) float srows[kMaxSrcSmem * kHeadDim];   // unit-norm source keys
     const int unit = blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
-    const T *Kh = K + b * d.ks[0] + (long long)h * d.ks[1];
+    const T *Kh = K + b * ks.v[0] + (long long)h * ks.v[1];
+    const T *Sh = S + b * ss.v[0] + (long long)h * ss.v[1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int j0 = blockIdx.x * kSimChunk;
     const int j1 = min(j0 + kSimChunk, d.N);
@@ -32,7 +40,7 @@ __global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *
         // one warp per source row: load, normalise, store
         for (int a = warp; a < na; a += kSimThreads / 32) {
             const int i = src[(long long)unit * d.K_src + a0 + a];
-            const T *kp = Kh + (long long)i * d.ks[2] + lane * 4;
+            const T *kp = Sh + (long long)i * ss.v[2] + lane * 4;
             float v[4];
             if constexpr (sizeof(T) == 2) {
                 const uint2 raw = *reinterpret_cast<const uint2 *>(kp);
@@ -54,7 +62,7 @@ __global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *
 #pragma unroll
             for (int c = 0; c < kHeadDim / 8; ++c) {
                 float v[8];
-                load8(Kh + (long long)j * d.ks[2] + c * 8, v);
+                load8(Kh + (long long)j * ks.v[2] + c * 8, v);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     k[c * 8 + e] = v[e];
@@ -96,8 +104,8 @@ __global__ void decay_rounds_kernel(Dims d, const int *__restrict__ nbr_idx,
         for (int a = 0; a < d.K_src; ++a) {
             for (int u = threadIdx.x; u < d.m; u += blockDim.x) {
                 const int j = ni[a * d.m + u];
-                const float e = fmaxf(ne[a * d.m + u], 0.f);
-                s[j] = s[j] * (1.0f - d.lambda * e);
+                s[j] = d.signal == GRAPHKV_SIGNAL_EVICT ? -INFINITY
+                                                        : s[j] * signal_factor(ne[a * d.m + u], d.lambda, 1, d.signal);
             }
             __syncthreads();
         }

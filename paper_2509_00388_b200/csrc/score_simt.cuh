@@ -155,9 +155,9 @@ __global__ void __launch_bounds__(kEmitThreads) score_emit_simt(Dims d, const T 
     }
 }
 
-// 1-D max pooling, stride 1, same length; positions outside [0,N) are ignored.
-// grid (ceil(N/256), units), block 256.
-__global__ void pool_max_kernel(int N, int kp, const float *__restrict__ a,
+// 1-D pooling, stride 1, same length: the maximum over the positions inside [0,N), or (avg) the
+// sum over them divided by kp (zeros outside the row).  grid (ceil(N/256), units), block 256.
+__global__ void pool_max_kernel(int N, int kp, int avg, const float *__restrict__ a,
                                 float *__restrict__ s)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -166,7 +166,12 @@ __global__ void pool_max_kernel(int N, int kp, const float *__restrict__ a,
     const int half = (kp - 1) / 2;
     const int lo = max(j - half, 0), hi = min(j + half, N - 1);
     float best = row[lo];
-    for (int t = lo + 1; t <= hi; ++t) best = fmaxf(best, row[t]);
+    if (avg) {
+        for (int t = lo + 1; t <= hi; ++t) best += row[t];
+        best /= (float)kp;
+    } else {
+        for (int t = lo + 1; t <= hi; ++t) best = fmaxf(best, row[t]);
+    }
     s[(long long)blockIdx.y * N + j] = best;
 }
 

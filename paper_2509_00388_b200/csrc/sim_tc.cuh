@@ -33,7 +33,9 @@ constexpr int kMaxBins = 256;           // cosine bins over [-1, 1] for the per-
 
 struct SimTcArgs {
     Dims d;
-    const __nv_bfloat16 *K;
+    const __nv_bfloat16 *S;   // tensor the source nodes' vectors are read from (the swept tensor comes
+                              // through the tensor map)
+    long long ss[3];          // its element strides: batch, head, token
     const int *src;        // [units][K_src] source positions
     Cand *cand;            // [units][K_src][chunks][kCandCap]; unused slots hold e = kCandEmpty
     uint32_t *cand_hist;   // [units][K_src][kCandBins] listed edges per cosine bin (zeroed before)
@@ -115,7 +117,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     const int per = a.n_tiles / a.chunks, rem = a.n_tiles % a.chunks;
     const int t0 = chunk * per + min(chunk, rem);
     const int n_local = per + (chunk < rem ? 1 : 0);
-    const __nv_bfloat16 *Kh = a.K + b * d.ks[0] + (long long)h * d.ks[1];
+    const __nv_bfloat16 *Sh = a.S + b * a.ss[0] + (long long)h * a.ss[1];
     const int *src = a.src + (long long)unit * d.K_src;
 
     int n_ahead = 0;                 // tiles thread 0 has requested before the roles split
@@ -155,7 +157,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         int pos = -1;
         if (in && r < d.K_src) {
             pos = src[r];
-            v = *reinterpret_cast<const uint4 *>(Kh + (long long)pos * d.ks[2] + c16 * 8);
+            v = *reinterpret_cast<const uint4 *>(Sh + (long long)pos * a.ss[2] + c16 * 8);
         }
         if (in) *reinterpret_cast<uint4 *>(gen + sw128_offset(NP, r, c16)) = v;
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};

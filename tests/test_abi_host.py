@@ -35,8 +35,8 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_params_struct_matches_header_size():
-    # 14 four-byte fields + 9 int64 strides
-    assert C.sizeof(gk.Params) == 14 * 4 + 9 * 8
+    # 14 four-byte fields + 9 int64 strides + 2 four-byte fields
+    assert C.sizeof(gk.Params) == 14 * 4 + 9 * 8 + 2 * 4
 
 
 def _params(**kw):

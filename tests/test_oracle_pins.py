@@ -444,3 +444,115 @@ def test_decay_changes_selection_away_from_duplicates():
     assert idx0[0, 0].tolist() == [2, 3, 4]
     assert 2 in idx1[0, 0].tolist() and 3 not in idx1[0, 0].tolist() and 4 not in idx1[0, 0].tolist()
     assert s1[0, 0, 3].item() == 0.0 and s1[0, 0, 4].item() == 0.0
+
+
+# ----------------------------------------------------------------------------- KNorm initial score
+
+
+def test_knorm_score_is_the_reciprocal_key_norm_of_the_prefix():
+    rng = np.random.default_rng(3)
+    K = torch.from_numpy(rng.standard_normal((2, 2, 37 + 5, 16)).astype(np.float32) * 3)
+    K[0, 1, 4] = 0.0                                   # a zero key: norm floored, score finite
+    s = okv.score_knorm(K, window=5)
+    assert s.shape == (2, 2, 37)
+    want = 1.0 / np.maximum(np.linalg.norm(K[:, :, :37].double().numpy(), axis=-1), 1e-12)
+    np.testing.assert_allclose(s.double().numpy(), want, rtol=1e-6)
+    assert np.isfinite(s.numpy()).all() and (s.numpy() > 0).all()
+    # ranks like ascending L2 norm: the key of lowest norm scores highest
+    norms = np.linalg.norm(K[1, 0, :37].double().numpy(), axis=-1)
+    assert int(s[1, 0].argmax()) == int(norms.argmin())
+    # scaling a key by c scales its score by 1/c
+    K2 = K.clone()
+    K2[1, 1, 7] *= 4.0
+    assert abs(okv.score_knorm(K2, 5)[1, 1, 7].item() * 4.0 - s[1, 1, 7].item()) < 1e-6
+
+
+# ----------------------------------------------------------------------------- variants
+
+
+def test_average_pooling_matches_the_library_routine():
+    # mean over kp positions with zeros outside the row = avg_pool1d with zero padding counted
+    for seed, (G, W, D, N, kp) in enumerate([(2, 4, 16, 40, 7), (1, 3, 8, 9, 5), (2, 2, 8, 30, 1)]):
+        Qg, Kh = rand_unit(seed, G, W, D, N, scale=2.0)
+        a, s = okv.score_unit(Qg, Kh, pool_kernel=kp, pool_mode=okv.POOL_AVG)
+        ref = torch.nn.functional.avg_pool1d(a[None, None], kp, stride=1, padding=kp // 2,
+                                             count_include_pad=True)[0, 0]
+        np.testing.assert_allclose(s.double().numpy(), ref.numpy(), rtol=1e-6)
+        assert s.shape[0] == N
+    # and through the whole-layer driver
+    Qw, K, V = _tiny_inputs(seed=4)
+    s_avg = okv.score(Qw, K, 4, 5, pool_mode=okv.POOL_AVG)
+    _, su = okv.score_unit(Qw[1, 2:4], K[1, 1], 5, pool_mode=okv.POOL_AVG)
+    assert torch.equal(su, s_avg[1, 1])
+    assert not torch.equal(s_avg, okv.score(Qw, K, 4, 5))
+
+
+def brute_propagate(S, A, s, N, k, m, T, lam, signal=0, reselect=False):
+    """Eq. 1-5 by definition in numpy fp64: sources = top-k, edges = cosine(S[i], A[j]),
+    neighbourhoods = top-m (j != i), T rounds; with reselect the graph is rebuilt every round from
+    the scores rounded to fp32."""
+    S = S.double().numpy()[:N]
+    A = A.double().numpy()[:N]
+    Sn = S / np.maximum(np.linalg.norm(S, axis=1, keepdims=True), 1e-12)
+    An = A / np.maximum(np.linalg.norm(A, axis=1, keepdims=True), 1e-12)
+    cos = np.clip(Sn @ An.T, -1.0, 1.0)
+    cur = s.double().numpy().copy()
+
+    def graph(scores32):
+        src = brute_topk(scores32, k)
+        return src, [brute_topk(cos[i].astype(np.float32), m, skip=i) for i in src]
+
+    src, nbrs = graph(cur.astype(np.float32))
+    for t in range(T):
+        if reselect and t > 0:
+            cur = cur.astype(np.float32).astype(np.float64)
+            src, nbrs = graph(cur.astype(np.float32))
+        for i, nb in zip(src, nbrs):
+            for j in nb:
+                e = max(cos[i, j], 0.0)
+                if signal == 2:
+                    cur[j] = -np.inf
+                elif signal == 1:
+                    cur[j] *= 1.0 + lam * e
+                else:
+                    cur[j] *= 1.0 - lam * e
+    return cur.astype(np.float32), src
+
+
+@pytest.mark.parametrize("signal", [0, 1, 2])
+@pytest.mark.parametrize("reselect", [0, 1])
+def test_signals_and_reselection_match_the_definition(signal, reselect):
+    rng = np.random.default_rng(10 * signal + reselect)
+    N, W, D = 60, 2, 8
+    K = torch.from_numpy(rng.standard_normal((1, 1, N + W, D)).astype(np.float32))
+    s0 = torch.from_numpy(rng.random((1, 1, N)).astype(np.float32) + 0.1)
+    got, src = okv.propagate(K, s0, W, 4, 3, 3, 0.7, signal=signal, reselect=reselect)
+    want, want_src = brute_propagate(K[0, 0], K[0, 0], s0[0, 0], N, 4, 3, 3, 0.7, signal, bool(reselect))
+    g, w = got[0, 0].numpy(), want
+    assert np.array_equal(np.isinf(g), np.isinf(w))
+    np.testing.assert_allclose(g[np.isfinite(g)], w[np.isfinite(w)], rtol=1e-6)
+    assert sorted(src[0, 0].tolist()) == sorted(want_src.tolist())
+    if signal == 1:
+        assert np.all(g >= s0[0, 0].numpy())           # an enhanced signal never lowers a score
+    if signal == 2:
+        assert np.isinf(g).sum() > 0 and np.all(g[np.isfinite(g)] == s0[0, 0].numpy()[np.isfinite(g)])
+    if reselect:
+        # re-picking matters: some round takes other sources than the first
+        fixed, _ = okv.propagate(K, s0, W, 4, 3, 3, 0.7, signal=signal, reselect=0)
+        assert signal == 1 or not torch.equal(fixed, got)
+
+
+def test_value_and_key_value_edges_match_the_definition():
+    rng = np.random.default_rng(7)
+    N, W, D = 50, 2, 8
+    K = torch.from_numpy(rng.standard_normal((N + W, D)).astype(np.float32))
+    V = torch.from_numpy(rng.standard_normal((N + W, D)).astype(np.float32))
+    s0 = torch.from_numpy(rng.random(N).astype(np.float32) + 0.1)
+    for S, A in ((V, V), (K, V)):
+        got, src, nbr, nbr_e = okv.propagate_unit(A, s0, N, 3, 4, 2, 0.5, Sh=S)
+        want, want_src = brute_propagate(S, A, s0, N, 3, 4, 2, 0.5)
+        np.testing.assert_allclose(got.numpy(), want, rtol=1e-6)
+        assert sorted(src.tolist()) == sorted(want_src.tolist())
+        i = int(src[0])
+        np.testing.assert_allclose(
+            okv.edges_unit(A, N, i, Sh=S).numpy()[nbr[0].numpy()], nbr_e[0].numpy(), rtol=1e-12)
