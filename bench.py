@@ -488,11 +488,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-secondary", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's number of sequences")
+    ap.add_argument("--topk-nodes", type=int, default=0, help="override the workload's number of source nodes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = wl.CONFIGS[args.workload]
     if args.batch > 0:
         cfg = wl.scaled(cfg, batch=args.batch, name=f"{cfg.name}[batch={args.batch}]")
+    if args.topk_nodes > 0:
+        cfg = wl.scaled(cfg, topk_nodes=args.topk_nodes, name=f"{cfg.name}[topk_nodes={args.topk_nodes}]")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -47,18 +47,19 @@ struct Smem {
     uint32_t *misc;       // [32] broadcast words and this CTA's published counts
     int *st_idx;          // [kStage] staging: neighbour positions / candidate positions / survivors
     float *st_f;          // [kStage] staging: decay factors / survivors
-    int *nb_j;            // [kStage] the unit's neighbour lists, positions (every CTA holds a copy)
-    float *nb_f;          // [kStage] their decay factors over all rounds
+    int *nb_j;            // [stage_cap] the unit's neighbour lists, positions (every CTA holds a copy)
+    float *nb_f;          // [stage_cap] their decay factors over all rounds
+    int stage_cap;        // words of each of the four staging arrays (at least kStage)
     float *vals;          // [halo + chunk + halo]
 };
 
-__host__ __device__ inline size_t smem_bytes(int chunk, int halo)
+__host__ __device__ inline size_t smem_bytes(int chunk, int halo, int stage_cap = kStage)
 {
-    return (size_t)(kBins + kTotWords + kFineBins + 2 * kWarps + 32 + 4 * kStage) * 4 +
+    return (size_t)(kBins + kTotWords + kFineBins + 2 * kWarps + 32 + 4 * stage_cap) * 4 +
            (size_t)(chunk + 2 * halo + 8) * 4;
 }
 
-__device__ __forceinline__ Smem carve(uint8_t *raw, int halo)
+__device__ __forceinline__ Smem carve(uint8_t *raw, int halo, int stage_cap = kStage)
 {
     Smem s;
     s.hist = reinterpret_cast<uint32_t *>(raw);
@@ -67,10 +68,11 @@ __device__ __forceinline__ Smem carve(uint8_t *raw, int halo)
     s.wcnt = s.fine + kFineBins;
     s.misc = s.wcnt + 2 * kWarps;
     s.st_idx = reinterpret_cast<int *>(s.misc + 32);
-    s.st_f = reinterpret_cast<float *>(s.st_idx + kStage);
-    s.nb_j = reinterpret_cast<int *>(s.st_f + kStage);
-    s.nb_f = reinterpret_cast<float *>(s.nb_j + kStage);
-    s.vals = s.nb_f + kStage;
+    s.st_f = reinterpret_cast<float *>(s.st_idx + stage_cap);
+    s.nb_j = reinterpret_cast<int *>(s.st_f + stage_cap);
+    s.nb_f = reinterpret_cast<float *>(s.nb_j + stage_cap);
+    s.vals = s.nb_f + stage_cap;
+    s.stage_cap = stage_cap;
     (void)halo;
     return s;
 }
@@ -957,6 +959,7 @@ struct FinishArgs {
     const unsigned char *K, *V;
     unsigned char *K_out, *V_out;
     int wait_prior;            // launched with programmatic stream serialization
+    int stage_cap;             // words of each staging array in shared memory (K_src * m when it fits)
 };
 
 // Chunk [base, base + n_local) of a unit's scores into shared memory; returns `vals` with
@@ -1055,10 +1058,10 @@ __device__ void apply_lists(const Smem &s, float *vals, int base, int n_local, i
                             bool evict)
 {
     const int tid = threadIdx.x;
-    const int pairs = K_src * m;                           // <= kStage, so K_src <= kStage
+    const int pairs = K_src * m;                           // fits the staging arrays
     uint32_t *cnt = s.fine;                                // [4096] edges per table slot
-    uint32_t *src_mask = s.fine + 4096;                    // [kStage / 32] sources with a contested edge
-    for (int i = tid; i < 4096 + kStage / 32; i += kThreads) cnt[i] = 0u;
+    uint32_t *src_mask = s.fine + 4096;                    // [K_src / 32] sources with a contested edge
+    for (int i = tid; i < 4096 + (K_src + 31) / 32; i += kThreads) cnt[i] = 0u;
     __syncthreads();
     for (int p = tid; p < pairs; p += kThreads) {
         const int j = s.nb_j[p] - base;
@@ -1104,7 +1107,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     const Dims &d = a.d;
     const int C = a.C, R = a.R, rank = C > 1 ? (int)cl.block_rank() : 0;
     const int unit = a.unit0 + blockIdx.x / C;
-    const Smem s = carve(cs_smem, 0);
+    const Smem s = carve(cs_smem, 0, a.stage_cap);
     const int N = d.N, tid = threadIdx.x;
     const bool holds = rank < R;                           // this CTA keeps a chunk of the row
     const int base = rank * a.chunk;
@@ -1161,43 +1164,46 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
         int *ni = a.nbr_idx + (long long)unit * d.K_src * d.m;
         float *ne = a.nbr_e + (long long)unit * d.K_src * d.m;
         const int pairs = d.K_src * d.m;
-        if (pairs <= kStage) {
-            // Eq. 3, then Eq. 5 over the fixed graph with the T rounds folded into a power: the
-            // CTAs that hold the row get the unit's lists as (position, factor) in shared memory
-            if (a.merge) {
-                // the four warps of group g of merging rank r take sources (g + kMergeWarps * t) * M + r;
-                // a first CTA that holds the whole row leaves the merging to the others
-                const int warp = tid >> 5, grp = warp >> 2, wg = warp & 3;
-                Cand *surv = reinterpret_cast<Cand *>(s.st_idx) + grp * kSurvCap;
-                int *ns_sh = reinterpret_cast<int *>(s.misc) + 8 + grp;
-                const bool spare_first = R == 1 && C > 1;
-                const int M = spare_first ? C - 1 : C, mr = spare_first ? rank - 1 : rank;
-                for (int src = grp * M + mr; mr >= 0 && src < d.K_src; src += kMergeWarps * M) {
-                    const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
-                    const PushLists push{C, R, s.nb_j, s.nb_f, src * d.m, d.lambda, d.T, d.signal};
-                    merge_neighbours(cl, a.cand + slot * kCandCap,
-                                     a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
-                                     a.cand_chunks, d.m, surv, ns_sh, 1 + grp, wg, ni + src * d.m,
-                                     ne + src * d.m, push);
-                }
-                pc.mark();
-                if (C > 1) cl.sync(); else __syncthreads();       // every list has arrived
-                pc.mark();
-            } else if (holds) {
-                for (int i = tid; i < pairs; i += kThreads) {
-                    s.nb_j[i] = __ldcg(ni + i);
-                    s.nb_f[i] = signal_factor(__ldcg(ne + i), d.lambda, d.T, d.signal);
-                }
-                __syncthreads();
+        const bool staged = pairs <= s.stage_cap;          // the lists fit the shared-memory staging
+        // Eq. 3, then Eq. 5 over the fixed graph with the T rounds folded into a power: the
+        // CTAs that hold the row get the unit's lists as (position, factor) in shared memory
+        if (a.merge) {
+            // the four warps of group g of merging rank r take sources (g + kMergeWarps * t) * M + r;
+            // a first CTA that holds the whole row leaves the merging to the others
+            const int warp = tid >> 5, grp = warp >> 2, wg = warp & 3;
+            Cand *surv = reinterpret_cast<Cand *>(s.st_idx) + grp * kSurvCap;
+            int *ns_sh = reinterpret_cast<int *>(s.misc) + 8 + grp;
+            const bool spare_first = R == 1 && C > 1;
+            const int M = spare_first ? C - 1 : C, mr = spare_first ? rank - 1 : rank;
+            for (int src = grp * M + mr; mr >= 0 && src < d.K_src; src += kMergeWarps * M) {
+                const long long slot = ((long long)unit * d.K_src + src) * a.cand_chunks;
+                const PushLists push{C, staged ? R : 0, s.nb_j, s.nb_f, src * d.m, d.lambda, d.T, d.signal};
+                merge_neighbours(cl, a.cand + slot * kCandCap,
+                                 a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
+                                 a.cand_chunks, d.m, surv, ns_sh, 1 + grp, wg, ni + src * d.m,
+                                 ne + src * d.m, push);
             }
+            pc.mark();
+            if (!staged) __threadfence();                     // the lists are read back from global memory
+            if (C > 1) cl.sync(); else __syncthreads();       // every list has arrived
+            pc.mark();
+        } else if (staged && holds) {
+            for (int i = tid; i < pairs; i += kThreads) {
+                s.nb_j[i] = __ldcg(ni + i);
+                s.nb_f[i] = signal_factor(__ldcg(ne + i), d.lambda, d.T, d.signal);
+            }
+            __syncthreads();
+        }
+        if (staged) {
             if (holds) apply_lists(s, vals, base, n_local, d.K_src, d.m, d.signal == GRAPHKV_SIGNAL_EVICT);
         } else if (holds) {
             for (int src = 0; src < d.K_src; ++src) {
                 for (int u = tid; u < d.m; u += kThreads) {
-                    const int j = ni[src * d.m + u] - base;
+                    const int j = __ldcg(ni + src * d.m + u) - base;
                     if (j >= 0 && j < n_local)
                         vals[j] = d.signal == GRAPHKV_SIGNAL_EVICT
-                                      ? -INFINITY : vals[j] * signal_factor(ne[src * d.m + u], d.lambda, d.T, d.signal);
+                                      ? -INFINITY
+                                      : vals[j] * signal_factor(__ldcg(ne + src * d.m + u), d.lambda, d.T, d.signal);
                 }
                 __syncthreads();
             }

@@ -21,6 +21,7 @@ using namespace graphkv;
 namespace {
 
 constexpr size_t kAlign = 256;
+constexpr size_t kMaxSmem = 227 * 1024;      // dynamic shared memory a CTA may ask for
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Workspace carve-up; every region starts 256-byte aligned.
@@ -174,10 +175,12 @@ ClusterPlan cluster_plan(const Dims &d)
     return p;
 }
 
-// Tensor-core similarity sweep: usable for bf16 keys, up to 64 sources and 32 neighbours.
+// Tensor-core similarity sweep: usable for bf16 keys and up to 32 neighbours; 64 sources per
+// sweep of the keys, so a head with more sources (the paper's 0.3 x budget) is swept several times.
+constexpr int kSimMaxSources = 4096;
 struct SimPlan {
     bool ok;
-    int NP;         // source count padded to 16, 32 or 64
+    int NP;         // sources per sweep padded to 16, 32 or 64
     int chunks;     // CTAs (key chunks) per unit
     int n_tiles;    // 128-key tiles per unit
     int stages;
@@ -186,7 +189,7 @@ struct SimPlan {
 SimPlan sim_plan(const Dims &d, bool bf16)
 {
     SimPlan p{false, 16, 1, ceil_div(d.N, tc::kTileKeys), 5};
-    if (!bf16 || d.K_src < 1 || d.K_src > 64 || d.m < 1 || d.m > tc::kSimMaxNeighbors) return p;
+    if (!bf16 || d.K_src < 1 || d.K_src > kSimMaxSources || d.m < 1 || d.m > tc::kSimMaxNeighbors) return p;
     if (env_int("GRAPHKV_FORCE_SIMT", 0)) return p;
     if (!cluster_plan(d).ok) return p;          // its candidate lists are merged by the cluster kernel
     p.NP = d.K_src <= 16 ? 16 : (d.K_src <= 32 ? 32 : 64);
@@ -507,7 +510,7 @@ graphkv_status launch_cluster(const char *name, void (*kern)(Args), Args args, i
     static std::mutex mu;
     static signed char state[64] = {};
     if (!once_per_device(mu, state, [] {
-        const size_t mx = cs::smem_bytes(cs::kMaxChunk, cs::kMaxHalo);
+        const size_t mx = kMaxSmem;
         return set_smem(cs::pool_select_kernel<1>, mx) && set_smem(cs::pool_select_kernel<2>, mx) &&
                   set_smem(cs::pool_select_kernel<4>, mx) && set_smem(cs::pool_select_kernel<8>, mx) &&
                   set_smem(cs::pool_select_kernel<16>, mx) && set_smem(cs::pool_select_kernel<32>, mx) &&
@@ -583,22 +586,24 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const EdgeOperands<T> &
         const int group = units_per_group(d);
         for (int u0 = 0; u0 < d.units; u0 += group) {
             const int nu = std::min(group, d.units - u0);
-            tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(eo.S), {eo.ss[0], eo.ss[1], eo.ss[2]}, src, at<Cand>(ws, l.cand),
-                             at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
-                             sp.n_tiles, sp.stages, 0, wait_cycles()};
-            sa.wait_prior = next_launch_is_dependent();
-            const dim3 grid(sp.chunks, nu), block(tc::kSimThreads);
-            graphkv_status rc;
-            if (sp.NP == 16)
-                rc = launch_ex("similarity_tc", tc::similarity_tc<16>, grid, block,
-                               tc::sim_smem_bytes<16>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
-            else if (sp.NP == 32)
-                rc = launch_ex("similarity_tc", tc::similarity_tc<32>, grid, block,
-                               tc::sim_smem_bytes<32>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
-            else
-                rc = launch_ex("similarity_tc", tc::similarity_tc<64>, grid, block,
-                               tc::sim_smem_bytes<64>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
-            if (rc != GRAPHKV_OK) return rc;
+            for (int src0 = 0; src0 < d.K_src; src0 += sp.NP) {
+                tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(eo.S), {eo.ss[0], eo.ss[1], eo.ss[2]}, src, at<Cand>(ws, l.cand),
+                                 at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
+                                 sp.n_tiles, sp.stages, 0, wait_cycles(), src0, std::min(sp.NP, d.K_src - src0)};
+                sa.wait_prior = next_launch_is_dependent();
+                const dim3 grid(sp.chunks, nu), block(tc::kSimThreads);
+                graphkv_status rc;
+                if (sp.NP == 16)
+                    rc = launch_ex("similarity_tc", tc::similarity_tc<16>, grid, block,
+                                   tc::sim_smem_bytes<16>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
+                else if (sp.NP == 32)
+                    rc = launch_ex("similarity_tc", tc::similarity_tc<32>, grid, block,
+                                   tc::sim_smem_bytes<32>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
+                else
+                    rc = launch_ex("similarity_tc", tc::similarity_tc<64>, grid, block,
+                                   tc::sim_smem_bytes<64>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
+                if (rc != GRAPHKV_OK) return rc;
+            }
         }
         return GRAPHKV_OK;
     }
@@ -646,9 +651,14 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const 
                           has_graph ? 1 : 0, has_graph && merge ? 1 : 0, at<Cand>(ws, l.cand),
                           at<uint32_t>(ws, l.cand_hist), sim_plan(d, d.bf16 != 0).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
                           static_cast<const unsigned char *>(K), static_cast<const unsigned char *>(V),
-                          static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0};
+                          static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0, cs::kStage};
+        // the neighbour lists of a unit are staged in shared memory when K_src * m entries fit
+        const int pairs = has_graph ? d.K_src * d.m : 0;
+        if (pairs > cs::kStage && cs::smem_bytes(fp.chunk, halo, (pairs + 255) & ~255) <= kMaxSmem)
+            fa.stage_cap = (pairs + 255) & ~255;
         const char *name = has_graph ? (do_select ? "decay_select_gather" : "decay_rounds") : "select_gather";
-        return launch_cluster(name, cs::finish_kernel, fa, d.units, fp.C, cs::smem_bytes(fp.chunk, halo), st);
+        return launch_cluster(name, cs::finish_kernel, fa, d.units, fp.C,
+                              cs::smem_bytes(fp.chunk, halo, fa.stage_cap), st);
     }
     if (a)
         GKV_LAUNCH("pool_max", st,

@@ -3,7 +3,7 @@
 // source's top-m neighbourhood (Eq. 3).  The edge matrix never leaves the SM.
 //
 // One CTA owns a chunk of at most 512 / NP key tiles of one head (NP = source count padded to
-// 16, 32 or 64).  Each 128-key tile arrives by TMA, one tcgen05.mma block computes its
+// 16, 32 or 64; a head with more sources is swept once per 64 of them).  Each 128-key tile arrives by TMA, one tcgen05.mma block computes its
 // 128 x NP dot products against the source keys into its own TMEM columns, and the epilogue
 // threads (thread = key) take the key's norm from the staged tile.  When the sweep is over the
 // chunk's whole edge block still sits in TMEM, and the CTA
@@ -46,6 +46,7 @@ struct SimTcArgs {
     int stages;
     int wait_prior;        // launched with programmatic stream serialization
     long long wait_cycles; // limit of every wait of the kernel, in clocks
+    int src0, n_src;       // this launch takes sources [src0, src0 + n_src) of every unit (n_src <= NP)
 };
 
 template <int NP> __host__ __device__ constexpr int sim_tiles_cap() { return 512 / NP; }
@@ -118,7 +119,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     const int t0 = chunk * per + min(chunk, rem);
     const int n_local = per + (chunk < rem ? 1 : 0);
     const __nv_bfloat16 *Sh = a.S + b * a.ss[0] + (long long)h * a.ss[1];
-    const int *src = a.src + (long long)unit * d.K_src;
+    const int *src = a.src + (long long)unit * d.K_src + a.src0;
+    const int n_src = a.n_src;                               // sources of this launch
 
     int n_ahead = 0;                 // tiles thread 0 has requested before the roles split
     if (threadIdx.x == 0) {
@@ -155,7 +157,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         const bool in = i < NP * 16;
         uint4 v = make_uint4(0, 0, 0, 0);
         int pos = -1;
-        if (in && r < d.K_src) {
+        if (in && r < n_src) {
             pos = src[r];
             v = *reinterpret_cast<const uint4 *>(Sh + (long long)pos * a.ss[2] + c16 * 8);
         }
@@ -285,7 +287,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                 for (int q = 0; q < 4; ++q) {
                     const int c = g * 4 + q;
                     int bin = 0;
-                    if (c < d.K_src && best[c] > -INFINITY) {
+                    if (c < n_src && best[c] > -INFINITY) {
                         const float e = fminf(fmaxf(best[c] * src_inv[c], -1.0f), 1.0f);
                         bin = min(max(static_cast<int>((e + 1.0f) * (kMaxBins / 2)), 0), kMaxBins - 1);
                     }
@@ -296,7 +298,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             asm volatile("bar.sync 1, 256;" ::: "memory");
             pc.mark();
             const int ew = warp - 2;
-            for (int g = ew; g * 4 < d.K_src; g += 8) {
+            for (int g = ew; g * 4 < n_src; g += 8) {
                 uint32_t w8[8];              // this lane's eight threads' bins of sources 4g .. 4g+3
                 {
                     const uint4 lo = *reinterpret_cast<const uint4 *>(max_bin + g * kSimEpiThreads + lane * 8);
@@ -321,7 +323,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                     for (int q = 0; q < 4; ++q)
                         if (n[q] >= d.m + 1) bstar[q] |= 1u << bit;
                 }
-                if (lane < 4 && g * 4 + lane < d.K_src) {
+                if (lane < 4 && g * 4 + lane < n_src) {
                     const uint32_t bs = lane == 0 ? bstar[0] : lane == 1 ? bstar[1] : lane == 2 ? bstar[2] : bstar[3];
                     tau[g * 4 + lane] = bs == 0 ? -1.0f : (float)bs * (2.0f / kMaxBins) - 1.0f;
                     tau_bin[g * 4 + lane] = (int)bs;
@@ -340,7 +342,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             float theta[NP];
 #pragma unroll
             for (int c = 0; c < NP; ++c) {
-                const float q = c < d.K_src ? (tau[c] - 2.4e-7f) / src_inv[c] : INFINITY;
+                const float q = c < n_src ? (tau[c] - 2.4e-7f) / src_inv[c] : INFINITY;
                 theta[c] = q - fabsf(q) * 2.4e-7f - 1e-30f;
             }
             // (branch-free, the store and the count under one predicate; a key past the end of the
@@ -386,7 +388,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             {
                 const bool lost = xchg[1] != 0;
                 asm volatile("bar.sync 1, 256;" ::: "memory");
-                for (int c = et; c < d.K_src; c += kSimEpiThreads) {
+                for (int c = et; c < n_src; c += kSimEpiThreads) {
                     if (lost) cnt[c] = kCandCap + 1;
                     if (cnt[c] > kCandCap) xchg[1] = 1;               // some list overflowed
                 }
@@ -395,7 +397,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             // 3. a list that outgrew its capacity: exact m-th largest (edge desc, position asc)
             const bool any_overflow = xchg[1] != 0;
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            for (int c = 0; c < d.K_src && any_overflow; ++c) {
+            for (int c = 0; c < n_src && any_overflow; ++c) {
                 if (cnt[c] <= kCandCap) continue;                 // uniform: shared memory value
                 unsigned long long t64 = 0ull;
                 const float sinv = src_inv[c];
@@ -431,20 +433,20 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             }
             pc.mark();
             // write the lists out (unused slots marked empty) and count the listed edges per bin
-            for (int idx = et; idx < d.K_src * kCandCap; idx += kSimEpiThreads) {
+            for (int idx = et; idx < n_src * kCandCap; idx += kSimEpiThreads) {
                 const int c = idx / kCandCap, q = idx % kCandCap;
-                const long long slot = ((long long)unit * d.K_src + c) * a.chunks + chunk;
+                const long long slot = ((long long)unit * d.K_src + a.src0 + c) * a.chunks + chunk;
                 Cand cd{kCandEmpty, -1};
                 if (q < min(cnt[c], kCandCap)) {
                     cd = list[c * kCandCap + q];
-                    atomicAdd(a.cand_hist + ((long long)unit * d.K_src + c) * kCandBins + cand_bin(cd.e), 1u);
+                    atomicAdd(a.cand_hist + ((long long)unit * d.K_src + a.src0 + c) * kCandBins + cand_bin(cd.e), 1u);
                 }
                 a.cand[slot * kCandCap + q] = cd;
             }
         } else {
             // a wait ran out: publish empty lists so the merge reads nothing undefined
-            for (int i = et; i < d.K_src * kCandCap; i += kSimEpiThreads) {
-                const long long slot = ((long long)unit * d.K_src + i / kCandCap) * a.chunks + chunk;
+            for (int i = et; i < n_src * kCandCap; i += kSimEpiThreads) {
+                const long long slot = ((long long)unit * d.K_src + a.src0 + i / kCandCap) * a.chunks + chunk;
                 a.cand[slot * kCandCap + i % kCandCap] = Cand{kCandEmpty, -1};
             }
         }

@@ -242,14 +242,16 @@ def test_fallback_kernels_agree_with_the_oracle(gk, env):
 @pytest.mark.parametrize("case", [
     dict(topk_nodes=40, neighbors=12),                  # source count padded to 64
     dict(topk_nodes=64, neighbors=32),                  # the largest tensor-core similarity case
-    dict(topk_nodes=65, neighbors=8),                   # one more: generic similarity
+    dict(topk_nodes=65, neighbors=8),                   # one more: a second sweep for one source
+    dict(topk_nodes=154, neighbors=8, budget=512),      # 0.3 x budget, three sweeps of 64 sources
+    dict(topk_nodes=154, neighbors=32, budget=512, rounds=1),   # lists beyond the default staging
     dict(topk_nodes=12, neighbors=33),                  # neighbours above the candidate-list path
     dict(topk_nodes=12, neighbors=8, pool_kernel=131),  # pooling halo above the cluster kernel's
     dict(topk_nodes=3, neighbors=32, rounds=5, decay=0.5),
 ])
 def test_regime_boundaries(gk, case):
-    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=6100, budget=400, n_q_heads=8, n_kv_heads=2,
-                    n_clusters=48, **case)
+    cfg = wl.scaled(wl.LLAMA_32K, **{**dict(n_prefix=6100, budget=400, n_q_heads=8, n_kv_heads=2,
+                                            n_clusters=48), **case})
     check(gk, cfg, strict_overlap=False)
 
 
@@ -359,6 +361,13 @@ def test_full_llama_32k(gk):
 @pytest.mark.parametrize("layer", [0, 13, 31])
 def test_full_mistral_16k_layers(gk, layer):
     check(gk, wl.MISTRAL_16K, layer=layer)
+
+
+def test_full_mistral_16k_with_the_papers_source_count(gk):
+    # the source count the paper's ablation finds best: 0.3 x budget = 614 sources per head
+    cfg = wl.scaled(wl.MISTRAL_16K, topk_nodes=round(0.3 * wl.MISTRAL_16K.budget))
+    assert cfg.topk_nodes == 614
+    check(gk, cfg, layer=0)
 
 
 @pytest.mark.parametrize("layer", [0, 16, 31])
