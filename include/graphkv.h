@@ -186,6 +186,20 @@ graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, co
                                 float *scores_out, void *workspace, size_t workspace_bytes,
                                 void *stream);
 
+/* graphkv_compress for several layers (or sequences) of one shape with a budget each: the
+ * layer-specific k_l of the Problem Formulation, e.g. PyramidKV's budgets that shrink with depth.
+ * The batch dimension of the params enumerates the layers: layer i's Qw, K and V start i batch
+ * strides after the base pointers (a cache kept as one [layers][heads][L][D] allocation), and
+ * budgets[i] (a HOST array of params.batch entries, 1 <= budgets[i] <= params.budget) is its
+ * budget.  params.budget is the row capacity of the outputs: K_out / V_out are
+ * [batch][n_kv_heads][budget + W][D] and idx_out [batch][n_kv_heads][budget]; layer i fills its
+ * first budgets[i] (+ W) rows and leaves the rest untouched.  All layers run in one set of
+ * launches.  At most 64 layers per call (GRAPHKV_ERR_UNSUPPORTED beyond). */
+graphkv_status graphkv_compress_layers(const graphkv_params *params, const int32_t *budgets,
+                                       const void *Qw, const void *K, const void *V, void *K_out,
+                                       void *V_out, int32_t *idx_out, float *scores_out,
+                                       void *workspace, size_t workspace_bytes, void *stream);
+
 /* Synchronises `stream` and returns the status word kernels keep at the head of the workspace
  * (GRAPHKV_OK unless a bounded device-side wait ran out or a CUDA error surfaced).  The only
  * call that blocks the host. */

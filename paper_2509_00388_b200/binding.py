@@ -28,7 +28,7 @@ EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_scor
            "graphkv_read_status", "graphkv_status_string", "graphkv_launch_count",
            "graphkv_trace_enable", "graphkv_trace_read", "graphkv_builtin_scratch_needed",
            "graphkv_score_noalloc", "graphkv_read_status_noalloc", "graphkv_read_neighbors", "graphkv_phase_timing_read", "graphkv_score_knorm",
-           "graphkv_propagate_edges")
+           "graphkv_propagate_edges", "graphkv_compress_layers")
 
 
 class GraphKVError(RuntimeError):
@@ -77,6 +77,8 @@ def lib() -> C.CDLL:
         L.graphkv_select_gather.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.graphkv_compress.restype = C.c_int
         L.graphkv_compress.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.graphkv_compress_layers.restype = C.c_int
+        L.graphkv_compress_layers.argtypes = [P, C.POINTER(C.c_int32), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.graphkv_read_status.restype = C.c_int
         L.graphkv_read_status.argtypes = [vp, vp]
         L.graphkv_score_knorm.restype = C.c_int
@@ -230,6 +232,16 @@ def graphkv_compress(p: Params, Qw: torch.Tensor, K: torch.Tensor, V: torch.Tens
     _check(lib().graphkv_compress(C.byref(p), _ptr(Qw), _ptr(K), _ptr(V), _ptr(K_out),
                                   _ptr(V_out), _ptr(idx_out), _ptr(scores_out), _ptr(ws),
                                   ws.numel(), _stream(K.device)), "graphkv_compress")
+
+
+def graphkv_compress_layers(p: Params, budgets, Qw: torch.Tensor, K: torch.Tensor, V: torch.Tensor,
+                            K_out: torch.Tensor, V_out: torch.Tensor, idx_out: torch.Tensor,
+                            scores_out: Optional[torch.Tensor], ws: torch.Tensor) -> None:
+    """graphkv_compress with a budget per batch element (layer); p.budget is the outputs' capacity."""
+    arr = (C.c_int32 * p.batch)(*[int(b) for b in budgets])
+    _check(lib().graphkv_compress_layers(C.byref(p), arr, _ptr(Qw), _ptr(K), _ptr(V), _ptr(K_out),
+                                         _ptr(V_out), _ptr(idx_out), _ptr(scores_out), _ptr(ws),
+                                         ws.numel(), _stream(K.device)), "graphkv_compress_layers")
 
 
 def graphkv_read_status(ws: torch.Tensor) -> int:

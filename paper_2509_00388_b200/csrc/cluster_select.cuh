@@ -33,6 +33,7 @@ constexpr int kMaxPerThread = kMaxChunk / kThreads;
 constexpr int kStage = 2048;           // neighbour-list entries staged in shared memory at a time
 constexpr int kMergeWarps = 8;         // groups of four warps of a CTA, one source each at a time
 constexpr int kSurvCap = 256;          // merged candidates one warp ranks in shared memory
+constexpr int kMaxBudgets = 64;        // batch elements with a budget of their own per launch
 constexpr int kFineBins = 8192;        // one-pass selection: histogram over the top 13 bits of the ordered image
 constexpr int kFineShift = 19;
 constexpr int kTotWords = kFineBins / 2;   // a CTA's slice of the cluster-wide fine histogram (C >= 2)
@@ -960,6 +961,8 @@ struct FinishArgs {
     unsigned char *K_out, *V_out;
     int wait_prior;            // launched with programmatic stream serialization
     int stage_cap;             // words of each staging array in shared memory (K_src * m when it fits)
+    int per_batch_budget;      // budgets differ per batch element: budget_of[unit / hkv] (d.B: output rows)
+    int budget_of[kMaxBudgets];
 };
 
 // Chunk [base, base + n_local) of a unit's scores into shared memory; returns `vals` with
@@ -1121,7 +1124,8 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     pc.mark();
     const int b = unit / d.hkv, h = unit % d.hkv;
     const long long row_bytes = (long long)kHeadDim * a.elem_bytes;
-    const int rows_out = d.B + d.W;
+    const int rows_out = d.B + d.W;                        // rows the outputs hold per unit
+    const int B = a.per_batch_budget ? a.budget_of[b] : d.B;   // this unit's budget
     const int vpr = (int)(row_bytes >> 4);                 // 16-byte pieces per row
     const unsigned char *k0 = a.K ? a.K + (b * d.ks[0] + h * d.ks[1]) * a.elem_bytes : nullptr;
     const unsigned char *v0 = a.V ? a.V + (b * d.vs[0] + h * d.vs[1]) * a.elem_bytes : nullptr;
@@ -1211,7 +1215,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     }
     pc.mark();
     // the window rows do not depend on the selection (their loads return while the scores are stored)
-    if (gathers) copy_rows(d.B, (long long)d.W * 2 * vpr, [&](int t) { return (long long)(N + (t - d.B)); });
+    if (gathers) copy_rows(B, (long long)d.W * 2 * vpr, [&](int t) { return (long long)(N + (t - B)); });
     if ((a.a || a.has_graph) && holds) store_chunk(row_s + base, vals, n_local);
     pc.mark();
 
@@ -1223,15 +1227,15 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
             int *list = s.st_idx;
             // (a short chunk is ranked whole: the passes that list candidates would cost more,
             // and a budget above a sixteenth of the chunk leaves too many to gain anything)
-            const bool sparse = (long long)d.B * 16 <= a.chunk;
+            const bool sparse = (long long)B * 16 <= a.chunk;
             const int n_c = a.chunk >= 4 * kStage && sparse
-                                ? filter_candidates(s, vals, n_local, (uint32_t)d.B, list, 4 * kStage) : -1;
+                                ? filter_candidates(s, vals, n_local, (uint32_t)B, list, 4 * kStage) : -1;
             pc.mark();
             const RowView row{vals, n_c >= 0 ? list : nullptr, n_c >= 0 ? n_c : n_local};
             // a sparse selection takes the one-pass search, a dense one the digit-by-digit search
             // (its threshold bin would hold too many elements to rank by counting)
-            const Threshold th = sparse ? cluster_kth_fine(cl, R, rank, s, row, base, (uint32_t)d.B, pc)
-                                        : cluster_kth(cl, R, rank, s, row, (uint32_t)d.B);
+            const Threshold th = sparse ? cluster_kth_fine(cl, R, rank, s, row, base, (uint32_t)B, pc)
+                                        : cluster_kth(cl, R, rank, s, row, (uint32_t)B);
             cluster_emit_sorted(cl, R, rank, s, row, base, th, idx);
         }
         pc.mark();
@@ -1239,7 +1243,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
         if (C > 1) cl.sync(); else __syncthreads();
         pc.mark();
         // gather: the cluster's threads share the 16-byte pieces of the B kept rows
-        if (gathers) copy_rows(0, (long long)d.B * 2 * vpr, [&](int t) { return (long long)__ldcg(idx + t); });
+        if (gathers) copy_rows(0, (long long)B * 2 * vpr, [&](int t) { return (long long)__ldcg(idx + t); });
     }
     pc.mark();
     if (C > 1) cl.sync();      // no CTA leaves while its shared memory may still be read

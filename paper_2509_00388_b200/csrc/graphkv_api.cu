@@ -639,6 +639,9 @@ FinishPlan finish_plan(const Dims &d, int halo)
     return p;
 }
 
+// Per-batch-element budgets of the call in flight (graphkv_compress_layers), or none.
+thread_local const int32_t *t_budgets = nullptr;
+
 graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const float *a, float *s,
                           bool has_graph, bool merge, bool do_select, const void *K, const void *V,
                           void *K_out, void *V_out, int *idx_out, void *ws, cudaStream_t st)
@@ -651,7 +654,12 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const 
                           has_graph ? 1 : 0, has_graph && merge ? 1 : 0, at<Cand>(ws, l.cand),
                           at<uint32_t>(ws, l.cand_hist), sim_plan(d, d.bf16 != 0).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
                           static_cast<const unsigned char *>(K), static_cast<const unsigned char *>(V),
-                          static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0, cs::kStage};
+                          static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0, cs::kStage,
+                          0, {}};
+        if (t_budgets && do_select) {
+            fa.per_batch_budget = 1;
+            for (int i = 0; i < d.batch; ++i) fa.budget_of[i] = t_budgets[i];
+        }
         // the neighbour lists of a unit are staged in shared memory when K_src * m entries fit
         const int pairs = has_graph ? d.K_src * d.m : 0;
         if (pairs > cs::kStage && cs::smem_bytes(fp.chunk, halo, (pairs + 255) & ~255) <= kMaxSmem)
@@ -660,6 +668,7 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const 
         return launch_cluster(name, cs::finish_kernel, fa, d.units, fp.C,
                               cs::smem_bytes(fp.chunk, halo, fa.stage_cap), st);
     }
+    if (t_budgets && do_select) return GRAPHKV_ERR_UNSUPPORTED;      // only the cluster kernel takes budgets per layer
     if (a)
         GKV_LAUNCH("pool_max", st,
                    (pool_max_kernel<<<dim3(ceil_div(d.N, 256), d.units), 256, 0, st>>>(d.N, d.kp, d.pool_avg, a, s)));
@@ -1017,6 +1026,22 @@ graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, co
                            workspace, st);
     return do_compress(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), V, K_out,
                        V_out, idx_out, s, workspace, st);
+}
+
+graphkv_status graphkv_compress_layers(const graphkv_params *params, const int32_t *budgets,
+                                       const void *Qw, const void *K, const void *V, void *K_out,
+                                       void *V_out, int32_t *idx_out, float *scores_out,
+                                       void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!params || !budgets) return GRAPHKV_ERR_INVALID_ARG;
+    if (params->batch > cs::kMaxBudgets) return GRAPHKV_ERR_UNSUPPORTED;
+    for (int i = 0; i < params->batch; ++i)
+        if (budgets[i] < 1 || budgets[i] > params->budget) return GRAPHKV_ERR_INVALID_ARG;
+    t_budgets = budgets;
+    const graphkv_status rc = graphkv_compress(params, Qw, K, V, K_out, V_out, idx_out, scores_out,
+                                               workspace, workspace_bytes, stream);
+    t_budgets = nullptr;
+    return rc;
 }
 
 graphkv_status graphkv_read_status(const void *workspace, void *stream)

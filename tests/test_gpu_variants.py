@@ -216,3 +216,46 @@ def test_reselecting_sources_every_round(gk, env_simt, monkeypatch):
     _, _, o_idx, _ = okv.compress(inp["Qw"], inp["K"], inp["V"], reselect=1, **kwargs(cfg))
     common = sum(len(set(o_idx[0, h].tolist()) & set(idx2.cpu()[0, h].tolist())) for h in range(2))
     assert common >= 0.99 * 2 * cfg.budget
+
+
+def test_layers_with_their_own_budgets_in_one_call(gk):
+    # three layers stacked along the batch dimension, PyramidKV-style budgets; every layer must get
+    # exactly what a call of its own with its budget gives
+    cfg = small_cfg(batch=3, n_prefix=4200)
+    inp = wl.make_inputs(cfg)
+    Qd, Kd, Vd = (inp[k].to(DEV) for k in ("Qw", "K", "V"))
+    budgets = [300, 170, 64]
+    p = gk.make_params(Kd, Qw=Qd, V=Vd, **kwargs(cfg, budget=max(budgets)))
+    ws = gk.alloc_workspace(p, DEV)
+    K_out, V_out, idx, s = gk.alloc_outputs(p, Kd)
+    K_out.zero_(); V_out.zero_(); idx.fill_(-1)
+    gk.graphkv_compress_layers(p, budgets, Qd, Kd, Vd, K_out, V_out, idx, s, ws)
+    assert gk.graphkv_read_status(ws) == gk.OK
+    n = cfg.n_prefix
+    for i, b in enumerate(budgets):
+        # a call of its own for the layer: the same scores up to the rounding order of the sweeps'
+        # partial sums (their chunking depends on how many units a call holds)
+        pi = gk.make_params(Kd[i:i + 1], Qw=Qd[i:i + 1], V=Vd[i:i + 1], **kwargs(cfg, budget=b))
+        wsi = gk.alloc_workspace(pi, DEV)
+        Ko, Vo, io, so = gk.alloc_outputs(pi, Kd)
+        gk.graphkv_compress(pi, Qd[i:i + 1], Kd[i:i + 1], Vd[i:i + 1], Ko, Vo, io, so, wsi)
+        assert gk.graphkv_read_status(wsi) == gk.OK
+        assert pu.score_rel_err(s[i].cpu(), so[0].cpu()) <= 1e-5
+        rows = b + cfg.window
+        for h in range(cfg.n_kv_heads):
+            # the layer's own budget, selected exactly on the call's own scores; rows gathered bit for bit
+            want = np.sort(okv.topk(s[i, h].cpu(), b).numpy())
+            assert np.array_equal(idx[i, h, :b].cpu().numpy(), want)
+            ii = torch.from_numpy(want).long()
+            for out, X in ((K_out, inp["K"]), (V_out, inp["V"])):
+                ref = torch.cat([X[i, h, ii], X[i, h, n:]])
+                assert torch.equal(out[i, h, :rows].cpu().view(torch.int16), ref.view(torch.int16))
+        assert torch.all(idx[i, :, b:] == -1)
+        assert torch.all(K_out[i, :, rows:] == 0) and torch.all(V_out[i, :, rows:] == 0)
+        overlap = sum(len(set(idx[i, h, :b].tolist()) & set(io[0, h].tolist())) for h in range(cfg.n_kv_heads))
+        assert overlap >= 0.99 * b * cfg.n_kv_heads
+    bad = gk.lib().graphkv_compress_layers
+    import ctypes as C
+    arr = (C.c_int32 * 3)(300, 301, 64)
+    assert bad(C.byref(p), arr, Qd.data_ptr(), Kd.data_ptr(), Vd.data_ptr(), K_out.data_ptr(),
+               V_out.data_ptr(), idx.data_ptr(), None, ws.data_ptr(), ws.numel(), None) == gk.ERR_INVALID_ARG
