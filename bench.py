@@ -442,6 +442,42 @@ def measure_stacked(cfg, gk, dev, world, local, steps, warmup, blocks):
     return res
 
 
+def measure_decode(cfg, gk, dev, inp, peak):
+    """Decode-side micro-benchmark: one decoding step's attention over the full cache of the layer
+    and over the compact cache graphkv_compress leaves (B + W rows), same queries."""
+    Kd, Vd, Qd = inp["K"].to(dev), inp["V"].to(dev), inp["Qw"].to(dev)
+    p = gk.make_params(Kd, Qw=Qd, V=Vd, **cfg_kwargs(cfg))
+    ws = gk.alloc_workspace(p, dev)
+    K_out, V_out, idx, _ = gk.alloc_outputs(p, Kd, want_scores=False)
+    gk.graphkv_compress(p, Qd, Kd, Vd, K_out, V_out, idx, None, ws)
+    q = Qd[:, :, -1].contiguous()
+    out = {}
+    for name, (Kc, Vc) in {"full_cache": (Kd, Vd), "compact_cache": (K_out, V_out)}.items():
+        dp = gk.decode_params(q, Kc, Vc)
+        dws = gk.decode_workspace(dp, dev)
+        o = torch.empty((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.float32, device=dev)
+        flush = torch.empty(int(2.2 * L2_BYTES), dtype=torch.uint8, device=dev)
+        times = []
+        for _ in range(12):
+            flush.fill_(1)                                    # the cache comes from HBM every time
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            gk.graphkv_decode_attention(dp, q, Kc, Vc, o, dws)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            times.append(e0.elapsed_time(e1))
+        times = sorted(times[2:])
+        ms = times[len(times) // 2]
+        nbytes = 2 * Kc.numel() * Kc.element_size()
+        out[name] = {"rows": int(Kc.shape[2]), "ms": ms, "cache_bytes": nbytes,
+                     "achieved": nbytes / (ms * 1e-3) / 1e9, "unit": "GB/s",
+                     "frac": nbytes / (ms * 1e-3) / 1e9 / peak}
+    out["speedup"] = out["full_cache"]["ms"] / out["compact_cache"]["ms"]
+    out["note"] = ("attention of one decoding step, all query heads of the layer; L2 flushed before every "
+                   "call; median of 10")
+    return out
+
+
 def roofline_blocks(cfg, res, peak, peak_kind):
     """The dominant kernel's roofline entry, the whole path's, and every kernel's."""
     kernels = res["kernels"]
@@ -496,6 +532,9 @@ def run_ours(args, cfg):
     roofline, path, per = roofline_blocks(cfg, res, peak, peak_kind)
     inp = res.pop("host_inputs")
 
+    decode = None
+    if world == 1 and not args.no_secondary and cfg.n_layers == 1:
+        decode = measure_decode(cfg, gk, dev, inp, peak)
     secondary = None
     if world == 1 and not args.no_secondary and cfg.name != SECONDARY:
         cfg2 = wl.CONFIGS[SECONDARY]
@@ -536,7 +575,7 @@ def run_ours(args, cfg):
             "roofline": roofline, "roofline_path": path, "roofline_kernels": per,
             "cpu_baseline": cpu, "clocks": res["clocks"], "e2e": res["e2e"],
             "gpu_launches": res["launches"], "input_stats": res["input_stats"],
-            "secondary": secondary}
+            "decode": decode, "secondary": secondary}
     print(json.dumps(line))
 
 

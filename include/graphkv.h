@@ -200,6 +200,19 @@ graphkv_status graphkv_compress_layers(const graphkv_params *params, const int32
                                        void *V_out, int32_t *idx_out, float *scores_out,
                                        void *workspace, size_t workspace_bytes, void *stream);
 
+/* Decode-side micro-benchmark support (Efficiency Analysis: the paper's latency table is decoding
+ * latency; this is the attention of one decoding step over a cache, full or compact):
+ *   out[b][hq][:] = sum_j softmax_j(q[b][hq] . K[b][h][j] / sqrt(D)) * V[b][h][j],  h = hq / G,
+ * over params->seq_len rows of K and V per KV head (no mask: every cached row is visible to the
+ * new token).  q [batch][n_q_heads][D] with q_stride[0], q_stride[1]; K, V with k_stride,
+ * v_stride; out [batch][n_q_heads][D] fp32, dense.  Of the params only batch, n_q_heads,
+ * n_kv_heads, head_dim (128), seq_len, dtype and the strides are read; G <= 8.  The cache is read
+ * once.  Scratch: graphkv_decode_workspace_bytes(params) bytes. */
+size_t graphkv_decode_workspace_bytes(const graphkv_params *params);
+graphkv_status graphkv_decode_attention(const graphkv_params *params, const void *q, const void *K,
+                                        const void *V, float *out, void *workspace,
+                                        size_t workspace_bytes, void *stream);
+
 /* Synchronises `stream` and returns the status word kernels keep at the head of the workspace
  * (GRAPHKV_OK unless a bounded device-side wait ran out or a CUDA error surfaced).  The only
  * call that blocks the host. */

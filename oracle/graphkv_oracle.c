@@ -297,6 +297,36 @@ void okv_gather_unit(const unsigned char *Xh, int32_t N, int32_t W, size_t row_b
         memcpy(out + (size_t)(B + r) * row_bytes, Xh + (size_t)(N + r) * row_bytes, row_bytes);
 }
 
+/* ---- decode-side use of a cache: one new token's attention over `rows` cached rows ----------
+ * out[g][:] = sum_j softmax_j(q[g].K[j] / sqrt(D)) V[j] for the G query heads of one KV head
+ * (no mask: every cached row is visible).  q [G][D], Kh, Vh [rows][D]; out [G][D] fp64. */
+void okv_decode_attention_unit(const float *q, const float *Kh, const float *Vh, int32_t G,
+                               int32_t rows, int32_t D, double *out)
+{
+    double *l = (double *)malloc((size_t)rows * sizeof(double));
+    const double inv_sqrt_d = 1.0 / sqrt((double)D);
+    for (int32_t g = 0; g < G; ++g) {
+        double mx = -INFINITY;
+        for (int32_t j = 0; j < rows; ++j) {
+            double acc = 0.0;
+            for (int32_t d = 0; d < D; ++d) acc += (double)q[(size_t)g * D + d] * (double)Kh[(size_t)j * D + d];
+            l[j] = acc * inv_sqrt_d;
+            if (l[j] > mx) mx = l[j];
+        }
+        double z = 0.0;
+        for (int32_t j = 0; j < rows; ++j) {
+            l[j] = exp(l[j] - mx);
+            z += l[j];
+        }
+        for (int32_t d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int32_t j = 0; j < rows; ++j) acc += l[j] * (double)Vh[(size_t)j * D + d];
+            out[(size_t)g * D + d] = acc / z;
+        }
+    }
+    free(l);
+}
+
 /* ---- whole-layer drivers over contiguous [batch][heads][rows][D] arrays ------------------
  * Units are independent; OpenMP (when compiled in) only spreads units over cores. */
 int32_t okv_num_threads(void)

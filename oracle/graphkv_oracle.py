@@ -34,6 +34,7 @@ def lib() -> C.CDLL:
         _lib.okv_resolve_neighbors.restype = C.c_int32
         _lib.okv_num_threads.restype = C.c_int32
         for name in ("okv_topk", "okv_score_unit", "okv_score_knorm_unit", "okv_edges2_unit",
+                     "okv_decode_attention_unit",
                      "okv_propagate2_unit", "okv_propagate_reselect_unit", "okv_edges_unit", "okv_propagate_unit",
                      "okv_select_unit", "okv_gather_unit", "okv_score", "okv_propagate",
                      "okv_select_gather", "okv_compress"):
@@ -136,6 +137,24 @@ def score_knorm(K: torch.Tensor, window: int) -> torch.Tensor:
             kh = np.ascontiguousarray(k[bi, h])
             lib().okv_score_knorm_unit(_ptr(kh), C.c_int32(n), C.c_int32(d), _ptr(s[bi, h]))
     return torch.from_numpy(s)
+
+
+def decode_attention(q: torch.Tensor, K: torch.Tensor, V: torch.Tensor) -> torch.Tensor:
+    """One decoding step's attention over a cache: q [batch, n_q_heads, D], K and V
+    [batch, n_kv_heads, rows, D] -> fp64 [batch, n_q_heads, D]."""
+    b, hkv, rows, d = K.shape
+    g = q.shape[1] // hkv
+    qf, kf, vf = _f32(q), _f32(K), _f32(V)
+    out = np.empty((b, q.shape[1], d), dtype=np.float64)
+    for bi in range(b):
+        for h in range(hkv):
+            qq = np.ascontiguousarray(qf[bi, h * g:(h + 1) * g])
+            kk, vv = np.ascontiguousarray(kf[bi, h]), np.ascontiguousarray(vf[bi, h])
+            oo = np.empty((g, d), dtype=np.float64)
+            lib().okv_decode_attention_unit(_ptr(qq), _ptr(kk), _ptr(vv), C.c_int32(g), C.c_int32(rows),
+                                            C.c_int32(d), _ptr(oo))
+            out[bi, h * g:(h + 1) * g] = oo
+    return torch.from_numpy(out)
 
 
 def edges_unit(Kh: torch.Tensor, n_prefix: int, i: int,

@@ -28,7 +28,8 @@ EXPORTS = ("graphkv_workspace_bytes", "graphkv_resolve_neighbors", "graphkv_scor
            "graphkv_read_status", "graphkv_status_string", "graphkv_launch_count",
            "graphkv_trace_enable", "graphkv_trace_read", "graphkv_builtin_scratch_needed",
            "graphkv_score_noalloc", "graphkv_read_status_noalloc", "graphkv_read_neighbors", "graphkv_phase_timing_read", "graphkv_score_knorm",
-           "graphkv_propagate_edges", "graphkv_compress_layers")
+           "graphkv_propagate_edges", "graphkv_compress_layers", "graphkv_decode_workspace_bytes",
+           "graphkv_decode_attention")
 
 
 class GraphKVError(RuntimeError):
@@ -79,6 +80,10 @@ def lib() -> C.CDLL:
         L.graphkv_compress.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.graphkv_compress_layers.restype = C.c_int
         L.graphkv_compress_layers.argtypes = [P, C.POINTER(C.c_int32), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.graphkv_decode_workspace_bytes.restype = sz
+        L.graphkv_decode_workspace_bytes.argtypes = [P]
+        L.graphkv_decode_attention.restype = C.c_int
+        L.graphkv_decode_attention.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
         L.graphkv_read_status.restype = C.c_int
         L.graphkv_read_status.argtypes = [vp, vp]
         L.graphkv_score_knorm.restype = C.c_int
@@ -242,6 +247,31 @@ def graphkv_compress_layers(p: Params, budgets, Qw: torch.Tensor, K: torch.Tenso
     _check(lib().graphkv_compress_layers(C.byref(p), arr, _ptr(Qw), _ptr(K), _ptr(V), _ptr(K_out),
                                          _ptr(V_out), _ptr(idx_out), _ptr(scores_out), _ptr(ws),
                                          ws.numel(), _stream(K.device)), "graphkv_compress_layers")
+
+
+def decode_params(q: torch.Tensor, K: torch.Tensor, V: torch.Tensor) -> Params:
+    """Params of a decoding step: q [batch, n_q_heads, D], K and V [batch, n_kv_heads, rows, D]."""
+    p = Params()
+    p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = K.shape[0], q.shape[1], K.shape[1], K.shape[3]
+    p.seq_len, p.window, p.budget, p.pool_kernel = K.shape[2], 1, 1, 1
+    p.dtype = _dtype_code(K)
+    p.q_stride = (C.c_int64 * 3)(q.stride(0), q.stride(1), K.shape[3])
+    p.k_stride = _strides3(K)
+    p.v_stride = _strides3(V)
+    return p
+
+
+def graphkv_decode_attention(p: Params, q: torch.Tensor, K: torch.Tensor, V: torch.Tensor,
+                             out: torch.Tensor, ws: torch.Tensor) -> None:
+    _check(lib().graphkv_decode_attention(C.byref(p), _ptr(q), _ptr(K), _ptr(V), _ptr(out), _ptr(ws),
+                                          ws.numel(), _stream(K.device)), "graphkv_decode_attention")
+
+
+def decode_workspace(p: Params, device) -> torch.Tensor:
+    n = int(lib().graphkv_decode_workspace_bytes(C.byref(p)))
+    if n == 0:
+        raise GraphKVError(ERR_INVALID_ARG, "graphkv_decode_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
 
 
 def graphkv_read_status(ws: torch.Tensor) -> int:

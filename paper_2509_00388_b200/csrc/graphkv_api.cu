@@ -9,6 +9,7 @@
 
 #include "cluster_select.cuh"
 #include "common.cuh"
+#include "decode_attn.cuh"
 #include "gather.cuh"
 #include "propagate_simt.cuh"
 #include "score_simt.cuh"
@@ -1042,6 +1043,59 @@ graphkv_status graphkv_compress_layers(const graphkv_params *params, const int32
                                                workspace, workspace_bytes, stream);
     t_budgets = nullptr;
     return rc;
+}
+
+static bool decode_shape(const graphkv_params *p, DecodeArgs *a)
+{
+    if (!p || p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->seq_len < 1 ||
+        p->n_q_heads % p->n_kv_heads != 0 || p->head_dim != kHeadDim ||
+        p->n_q_heads / p->n_kv_heads > kDecMaxG || (long long)p->batch * p->n_kv_heads > 65535 ||
+        (p->dtype != GRAPHKV_BF16 && p->dtype != GRAPHKV_F32))
+        return false;
+    const int vec = p->dtype == GRAPHKV_BF16 ? 8 : 4;
+    for (int i = 0; i < 3; ++i)
+        if (p->k_stride[i] < 0 || p->v_stride[i] < 0 || p->k_stride[i] % vec || p->v_stride[i] % vec) return false;
+    if (p->q_stride[0] < 0 || p->q_stride[1] < kHeadDim) return false;
+    a->batch = p->batch; a->hq = p->n_q_heads; a->hkv = p->n_kv_heads; a->G = p->n_q_heads / p->n_kv_heads;
+    a->rows = p->seq_len;
+    const int units = p->batch * p->n_kv_heads;
+    const int tiles = ceil_div(p->seq_len, kDecTile);
+    a->splits = std::max(1, std::min(std::min(tiles, 256), ceil_div(4 * sm_count(), units)));
+    a->qs[0] = p->q_stride[0]; a->qs[1] = p->q_stride[1];
+    for (int i = 0; i < 3; ++i) { a->ks[i] = p->k_stride[i]; a->vs[i] = p->v_stride[i]; }
+    return true;
+}
+
+size_t graphkv_decode_workspace_bytes(const graphkv_params *params)
+{
+    DecodeArgs a;
+    if (!decode_shape(params, &a)) return 0;
+    return align_up((size_t)a.batch * a.hkv * a.splits * a.G * (2 + kHeadDim) * sizeof(float));
+}
+
+graphkv_status graphkv_decode_attention(const graphkv_params *params, const void *q, const void *K,
+                                        const void *V, float *out, void *workspace,
+                                        size_t workspace_bytes, void *stream)
+{
+    DecodeArgs a;
+    if (!decode_shape(params, &a)) return params && params->head_dim != kHeadDim ? GRAPHKV_ERR_UNSUPPORTED
+                                                                                  : GRAPHKV_ERR_INVALID_ARG;
+    if (!q || !K || !V || !out || !aligned16(K) || !aligned16(V)) return GRAPHKV_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < graphkv_decode_workspace_bytes(params)) return GRAPHKV_ERR_WORKSPACE;
+    a.part = static_cast<float *>(workspace);
+    a.out = out;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dim3 grid(a.splits, a.batch * a.hkv);
+    if (params->dtype == GRAPHKV_BF16)
+        GKV_LAUNCH("decode_partial", st, (decode_partial_kernel<__nv_bfloat16><<<grid, kDecThreads, 0, st>>>(
+                                             a, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(K),
+                                             static_cast<const __nv_bfloat16 *>(V))));
+    else
+        GKV_LAUNCH("decode_partial", st, (decode_partial_kernel<float><<<grid, kDecThreads, 0, st>>>(
+                                             a, static_cast<const float *>(q), static_cast<const float *>(K),
+                                             static_cast<const float *>(V))));
+    GKV_LAUNCH("decode_merge", st, (decode_merge_kernel<<<a.batch * a.hkv * a.G, kHeadDim, 0, st>>>(a)));
+    return launch_status();
 }
 
 graphkv_status graphkv_read_status(const void *workspace, void *stream)

@@ -259,3 +259,22 @@ def test_layers_with_their_own_budgets_in_one_call(gk):
     arr = (C.c_int32 * 3)(300, 301, 64)
     assert bad(C.byref(p), arr, Qd.data_ptr(), Kd.data_ptr(), Vd.data_ptr(), K_out.data_ptr(),
                V_out.data_ptr(), idx.data_ptr(), None, ws.data_ptr(), ws.numel(), None) == gk.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype,rows,hq,hkv,batch", [("bf16", 5000, 8, 2, 1), ("bf16", 37, 4, 4, 2),
+                                                     ("f32", 1300, 8, 1, 1), ("bf16", 544, 32, 8, 1)])
+def test_decode_attention_over_a_cache(gk, dtype, rows, hq, hkv, batch):
+    # one decoding step's attention over a cache of `rows` rows against the fp64 oracle
+    cfg = small_cfg(dtype=dtype, n_prefix=rows - 32, n_q_heads=hq, n_kv_heads=hkv, batch=batch)
+    inp = wl.make_inputs(cfg)
+    K, V = inp["K"], inp["V"]
+    q = inp["Qw"][:, :, -1].contiguous()                  # the last window query of every head
+    want = okv.decode_attention(q, K, V)
+    qd, Kd, Vd = q.to(DEV), K.to(DEV), V.to(DEV)
+    p = gk.decode_params(qd, Kd, Vd)
+    ws = gk.decode_workspace(p, DEV)
+    out = torch.empty((batch, hq, 128), dtype=torch.float32, device=DEV)
+    gk.graphkv_decode_attention(p, qd, Kd, Vd, out, ws)
+    torch.cuda.synchronize()
+    err = (out.cpu().double() - want).abs().max().item()
+    assert err <= 2e-3 * max(want.abs().max().item(), 1e-6), err

@@ -556,3 +556,19 @@ def test_value_and_key_value_edges_match_the_definition():
         i = int(src[0])
         np.testing.assert_allclose(
             okv.edges_unit(A, N, i, Sh=S).numpy()[nbr[0].numpy()], nbr_e[0].numpy(), rtol=1e-12)
+
+
+def test_decode_attention_matches_the_library_softmax():
+    rng = np.random.default_rng(5)
+    q = torch.from_numpy(rng.standard_normal((2, 4, 16)).astype(np.float32) * 2)
+    K = torch.from_numpy(rng.standard_normal((2, 2, 37, 16)).astype(np.float32))
+    V = torch.from_numpy(rng.standard_normal((2, 2, 37, 16)).astype(np.float32))
+    got = okv.decode_attention(q, K, V)
+    Kq = K.double().repeat_interleave(2, dim=1)            # KV head h serves query heads 2h, 2h+1
+    Vq = V.double().repeat_interleave(2, dim=1)
+    P = torch.softmax(torch.einsum("bhd,bhjd->bhj", q.double(), Kq) / 4.0, dim=-1)
+    want = torch.einsum("bhj,bhjd->bhd", P, Vq)
+    np.testing.assert_allclose(got.numpy(), want.numpy(), rtol=1e-12, atol=1e-14)
+    # one cached row: the output is that row's value
+    one = okv.decode_attention(q, K[:, :, :1], V[:, :, :1])
+    np.testing.assert_allclose(one[0, 3].numpy(), V[0, 1, 0].double().numpy(), rtol=1e-12)
