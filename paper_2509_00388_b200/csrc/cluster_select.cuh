@@ -86,12 +86,14 @@ struct Threshold {
 
 // The elements a selection ranks: all n of a chunk in shared memory (list == nullptr), or the n
 // of them whose chunk-relative positions `list` holds in ascending order.
+// (kListed as a template argument of the loops that walk a view keeps the unlisted case free of
+// the indirection.)
 struct RowView {
     const float *vals;
     const int *list;
     int n;
-    __device__ __forceinline__ int pos(int t) const { return list ? list[t] : t; }
-    __device__ __forceinline__ float at(int t) const { return vals[pos(t)]; }
+    template <bool kListed> __device__ __forceinline__ int pos(int t) const { return kListed ? list[t] : t; }
+    template <bool kListed> __device__ __forceinline__ float at(int t) const { return vals[pos<kListed>(t)]; }
 };
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane)
@@ -107,8 +109,9 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane)
 // k-th largest of the cluster's row.  vals: this CTA's chunk (n_local elements, shared memory).
 // All CTAs of the cluster call this with the same k (1 <= k <= elements in the row) and return
 // the same Threshold.  Executes the same number of cluster barriers in every CTA.
-__device__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const Smem &s,
-                                 const RowView &row, uint32_t k)
+template <bool kListed>
+__device__ Threshold cluster_kth_t(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                   const RowView &row, uint32_t k)
 {
     const int n_local = row.n;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -124,7 +127,7 @@ __device__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const S
             bool valid = i < n_local;
             uint32_t bin = 0;
             if (valid) {
-                const uint32_t u = float_to_key(row.at(i));
+                const uint32_t u = float_to_key(row.at<kListed>(i));
                 valid = (u & th.mask) == th.prefix;
                 bin = (u >> shift) & (nb - 1u);
             }
@@ -185,6 +188,12 @@ __device__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const S
         if (whole_class) break;       // every element of the threshold class is kept
     }
     return th;
+}
+
+__device__ __forceinline__ Threshold cluster_kth(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                                 const RowView &row, uint32_t k)
+{
+    return row.list ? cluster_kth_t<true>(cl, C, rank, s, row, k) : cluster_kth_t<false>(cl, C, rank, s, row, k);
 }
 
 // Candidates for the k largest of a chunk in shared memory.  The chunk's elements fall into
@@ -277,8 +286,9 @@ __device__ int filter_candidates(const Smem &s, const float *vals, int n_local, 
 // ranked by counting (value descending, position ascending), which gives the exact threshold
 // value and the number of its ties to keep.  Falls back to the three-digit search when b* holds
 // more than a few hundred elements (large budgets, rows with massive ties).  Same contract as cluster_kth.
-__device__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, const Smem &s,
-                                      const RowView &row, int base, uint32_t k, PhaseClock &pc)
+template <bool kListed>
+__device__ Threshold cluster_kth_fine_t(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                        const RowView &row, int base, uint32_t k, PhaseClock &pc)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_local = row.n;
@@ -288,7 +298,7 @@ __device__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, co
     for (int i0 = 0; i0 < n_local; i0 += kThreads) {
         const int i = i0 + tid;
         const bool valid = i < n_local;
-        const uint32_t bin = valid ? float_to_key(row.at(i)) >> kFineShift : 0u;
+        const uint32_t bin = valid ? float_to_key(row.at<kListed>(i)) >> kFineShift : 0u;
         // lanes sharing the first valid lane's bin are counted with one atomic (scores of a row
         // crowd into few bins); the others add for themselves
         const unsigned vm = __ballot_sync(0xffffffffu, valid);
@@ -368,7 +378,7 @@ __device__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, co
     const uint32_t bstar = s.misc[20], n_above = s.misc[21], n_in = s.misc[22];
     const uint32_t need = k - n_above;                   // of the n_in elements in bin b*
     if (need == n_in) return Threshold{bstar << kFineShift, (uint32_t)(kFineBins - 1) << kFineShift, n_in};
-    if (n_in > (uint32_t)kThreads / 4) return cluster_kth(cl, C, rank, s, row, k);     // too many to rank by counting
+    if (n_in > (uint32_t)kThreads / 4) return cluster_kth_t<kListed>(cl, C, rank, s, row, k);   // too many to rank by counting
     // this CTA's elements of bin b* -> its own lists (keys and positions in the two halves of hist):
     // every warp counts its own first, a scan over the warps gives each its slots
     uint32_t *ck = s.hist;
@@ -376,7 +386,7 @@ __device__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, co
     uint32_t mine_n = 0;
     for (int i0 = 0; i0 < n_local; i0 += kThreads) {
         const int i = i0 + tid;
-        const bool cand = i < n_local && (float_to_key(row.at(i)) >> kFineShift) == bstar;
+        const bool cand = i < n_local && (float_to_key(row.at<kListed>(i)) >> kFineShift) == bstar;
         mine_n += __popc(__ballot_sync(0xffffffffu, cand));
     }
     if (lane == 0) s.wcnt[warp] = mine_n;
@@ -394,7 +404,7 @@ __device__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, co
         bool cand = false;
         int at = 0;
         if (i < n_local) {
-            at = row.pos(i);
+            at = row.pos<kListed>(i);
             key = float_to_key(row.vals[at]);
             cand = (key >> kFineShift) == bstar;
         }
@@ -469,11 +479,19 @@ __device__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, co
     return Threshold{m0[18], 0xffffffffu, m0[19]};
 }
 
+__device__ __forceinline__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                                      const RowView &row, int base, uint32_t k, PhaseClock &pc)
+{
+    return row.list ? cluster_kth_fine_t<true>(cl, C, rank, s, row, base, k, pc)
+                    : cluster_kth_fine_t<false>(cl, C, rank, s, row, base, k, pc);
+}
+
 // Ascending positions of the kept elements of the cluster's row -> out[0..k).  Returns nothing;
 // ends with the writes of this CTA issued (callers fence before another CTA reads them).
 // One cluster barrier.
-__device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, const Smem &s,
-                                    const RowView &row, int base, Threshold th, int *out)
+template <bool kListed>
+__device__ void cluster_emit_sorted_t(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                      const RowView &row, int base, Threshold th, int *out)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_local = row.n;
@@ -485,7 +503,7 @@ __device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, cons
         const int i = i0 + lane;
         uint32_t mk = 0;
         const bool in = i < hi;
-        if (in) mk = float_to_key(row.at(i)) & th.mask;
+        if (in) mk = float_to_key(row.at<kListed>(i)) & th.mask;
         gt += __popc(__ballot_sync(0xffffffffu, in && mk > th.prefix));
         eq += __popc(__ballot_sync(0xffffffffu, in && mk == th.prefix));
     }
@@ -524,7 +542,7 @@ __device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, cons
         const bool in = i < hi;
         int at = 0;
         if (in) {
-            at = row.pos(i);
+            at = row.pos<kListed>(i);
             mk = float_to_key(row.vals[at]) & th.mask;
         }
         const bool is_gt = in && mk > th.prefix, is_eq = in && mk == th.prefix;
@@ -537,6 +555,13 @@ __device__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, cons
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
+}
+
+__device__ __forceinline__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, const Smem &s,
+                                                    const RowView &row, int base, Threshold th, int *out)
+{
+    if (row.list) cluster_emit_sorted_t<true>(cl, C, rank, s, row, base, th, out);
+    else cluster_emit_sorted_t<false>(cl, C, rank, s, row, base, th, out);
 }
 
 // The m largest edges (cosine descending, position ascending) of the lists when too many tie at
