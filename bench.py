@@ -472,6 +472,21 @@ def measure_decode(cfg, gk, dev, inp, peak):
         out[name] = {"rows": int(Kc.shape[2]), "ms": ms, "cache_bytes": nbytes,
                      "achieved": nbytes / (ms * 1e-3) / 1e9, "unit": "GB/s",
                      "frac": nbytes / (ms * 1e-3) / 1e9 / peak}
+    # the KNorm initial score: one pass over the prefix keys
+    sc = torch.empty((cfg.batch, cfg.n_kv_heads, cfg.n_prefix), dtype=torch.float32, device=dev)
+    times = []
+    for _ in range(12):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        gk.graphkv_score_knorm(p, Kd, sc)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        times.append(e0.elapsed_time(e1))
+    ms = sorted(times[2:])[5]
+    kb = cfg.batch * cfg.n_kv_heads * cfg.n_prefix * (cfg.head_dim * Kd.element_size() + 4)
+    out["knorm_score"] = {"ms": ms, "bytes": kb, "achieved": kb / (ms * 1e-3) / 1e9, "unit": "GB/s",
+                          "frac": kb / (ms * 1e-3) / 1e9 / peak}
     out["speedup"] = out["full_cache"]["ms"] / out["compact_cache"]["ms"]
     out["note"] = ("attention of one decoding step, all query heads of the layer; L2 flushed before every "
                    "call; median of 10")

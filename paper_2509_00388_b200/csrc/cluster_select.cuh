@@ -282,7 +282,7 @@ __device__ int filter_candidates(const Smem &s, const float *vals, int n_local, 
 // k-th largest of the cluster's row in one histogram pass: a kFineBins histogram over the top 13
 // bits of the ordered image (sign, exponent, four mantissa bits: sixteen bins per octave), reduced
 // across the cluster in slices; the bin b* that holds the k-th largest is located by every CTA
-// alike; the elements above it are kept, and the few inside it are pulled by the first CTA and
+// alike; the elements above it are kept, and the few inside it are pulled by every CTA and
 // ranked by counting (value descending, position ascending), which gives the exact threshold
 // value and the number of its ties to keep.  Falls back to the three-digit search when b* holds
 // more than a few hundred elements (large budgets, rows with massive ties).  Same contract as cluster_kth.
@@ -420,7 +420,11 @@ __device__ Threshold cluster_kth_fine_t(cg::cluster_group &cl, int C, int rank, 
     pc.mark();
     if (C > 1) cl.sync();                                // every CTA's list is complete
     pc.mark();
-    if (rank == 0) {
+    // every CTA pulls all lists (into the two halves of `tot`, idle by now) and ranks them itself:
+    // the same answer everywhere without another exchange
+    uint32_t *ak = s.tot;
+    int *ai = reinterpret_cast<int *>(s.tot + kThreads);
+    {
         uint32_t n_lane = 0;
         if (lane < C) n_lane = C > 1 ? cl.map_shared_rank(s.misc, lane)[17] : s.misc[17];
         uint32_t total = 0;
@@ -433,30 +437,23 @@ __device__ Threshold cluster_kth_fine_t(cg::cluster_group &cl, int C, int rank, 
             }
             total += n_p;
         }
-        uint32_t key = 0;
-        int pos = 0;
         if (mine_p >= 0) {
-            key = (C > 1 ? cl.map_shared_rank(ck, mine_p) : ck)[mine_j];
-            pos = (C > 1 ? cl.map_shared_rank(ci, mine_p) : ci)[mine_j];
-        }
-        __syncthreads();                                 // own list read before it is overwritten
-        if (mine_p >= 0) {
-            ck[tid] = key;
-            ci[tid] = pos;
+            ak[tid] = (C > 1 ? cl.map_shared_rank(ck, mine_p) : ck)[mine_j];
+            ai[tid] = (C > 1 ? cl.map_shared_rank(ci, mine_p) : ci)[mine_j];
         }
         __syncthreads();
         {
             // few candidates (at most kThreads / 4): four threads each, every one walking a quarter of the list
             const int t = tid >> 2, sub = tid & 3;
             const bool live = t < (int)total;
-            const uint32_t kt = live ? ck[t] : 0u;
-            const int pt = live ? ci[t] : 0;
+            const uint32_t kt = live ? ak[t] : 0u;
+            const int pt = live ? ai[t] : 0;
             uint32_t r = 0, n_gt = 0;                    // rank among all; candidates with a larger value
             if (live) {
 #pragma unroll 4
                 for (int u = sub; u < (int)total; u += 4) {
-                    const uint32_t ku = ck[u];
-                    const int pu = ci[u];
+                    const uint32_t ku = ak[u];
+                    const int pu = ai[u];
                     n_gt += ku > kt;
                     r += (ku > kt) | ((ku == kt) & (pu < pt));
                 }
@@ -473,10 +470,7 @@ __device__ Threshold cluster_kth_fine_t(cg::cluster_group &cl, int C, int rank, 
         __syncthreads();
     }
     pc.mark();
-    if (C > 1) cl.sync();                                // the first CTA's answer is published
-    pc.mark();
-    const uint32_t *m0 = C > 1 ? cl.map_shared_rank(s.misc, 0) : s.misc;
-    return Threshold{m0[18], 0xffffffffu, m0[19]};
+    return Threshold{s.misc[18], 0xffffffffu, s.misc[19]};
 }
 
 __device__ __forceinline__ Threshold cluster_kth_fine(cg::cluster_group &cl, int C, int rank, const Smem &s,
@@ -986,6 +980,7 @@ struct FinishArgs {
     unsigned char *K_out, *V_out;
     int wait_prior;            // launched with programmatic stream serialization
     int stage_cap;             // words of each staging array in shared memory (K_src * m when it fits)
+    int keep_scores;           // write the pooled / decayed scores back to `s` (0: nobody reads them)
     int per_batch_budget;      // budgets differ per batch element: budget_of[unit / hkv] (d.B: output rows)
     int budget_of[kMaxBudgets];
 };
@@ -1241,7 +1236,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     pc.mark();
     // the window rows do not depend on the selection (their loads return while the scores are stored)
     if (gathers) copy_rows(B, (long long)d.W * 2 * vpr, [&](int t) { return (long long)(N + (t - B)); });
-    if ((a.a || a.has_graph) && holds) store_chunk(row_s + base, vals, n_local);
+    if ((a.a || a.has_graph) && holds && a.keep_scores) store_chunk(row_s + base, vals, n_local);
     pc.mark();
 
     if (a.do_select) {

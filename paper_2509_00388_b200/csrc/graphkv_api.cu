@@ -642,6 +642,9 @@ FinishPlan finish_plan(const Dims &d, int halo)
 
 // Per-batch-element budgets of the call in flight (graphkv_compress_layers), or none.
 thread_local const int32_t *t_budgets = nullptr;
+// The caller of the call in flight wants the final scores (graphkv_compress without scores_out
+// does not: its last kernel then leaves them in shared memory).
+thread_local bool t_keep_scores = true;
 
 graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const float *a, float *s,
                           bool has_graph, bool merge, bool do_select, const void *K, const void *V,
@@ -656,7 +659,7 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const 
                           at<uint32_t>(ws, l.cand_hist), sim_plan(d, d.bf16 != 0).chunks, do_select ? 1 : 0, idx_out, elem_bytes,
                           static_cast<const unsigned char *>(K), static_cast<const unsigned char *>(V),
                           static_cast<unsigned char *>(K_out), static_cast<unsigned char *>(V_out), 0, cs::kStage,
-                          0, {}};
+                          (t_keep_scores || !do_select) ? 1 : 0, 0, {}};
         if (t_budgets && do_select) {
             fa.per_batch_budget = 1;
             for (int i = 0; i < d.batch; ++i) fa.budget_of[i] = t_budgets[i];
@@ -974,7 +977,8 @@ graphkv_status graphkv_score_knorm(const graphkv_params *params, const void *K, 
     if (!K || !scores || !aligned16(K)) return GRAPHKV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const long long rows = (long long)d.units * d.N;
-    const int blocks = (int)std::min<long long>((rows * 16 + 255) / 256, (long long)sm_count() * 16);
+    // one wave of resident CTAs (eight of 256 threads per SM), each group of 16 threads taking rows in steps
+    const int blocks = (int)std::min<long long>((rows * 16 + 255) / 256, (long long)sm_count() * 8);
     if (params->dtype == GRAPHKV_BF16)
         GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
                                           d, static_cast<const __nv_bfloat16 *>(K), scores)));
@@ -1021,12 +1025,15 @@ graphkv_status graphkv_compress(const graphkv_params *params, const void *Qw, co
     if ((rc = check_ws(l, workspace, workspace_bytes)) != GRAPHKV_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float *s = scores_out ? scores_out : at<float>(workspace, l.s);
+    t_keep_scores = scores_out != nullptr;
     if (params->dtype == GRAPHKV_BF16)
-        return do_compress(d, l, static_cast<const __nv_bfloat16 *>(Qw),
-                           static_cast<const __nv_bfloat16 *>(K), V, K_out, V_out, idx_out, s,
-                           workspace, st);
-    return do_compress(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), V, K_out,
-                       V_out, idx_out, s, workspace, st);
+        rc = do_compress(d, l, static_cast<const __nv_bfloat16 *>(Qw),
+                         static_cast<const __nv_bfloat16 *>(K), V, K_out, V_out, idx_out, s, workspace, st);
+    else
+        rc = do_compress(d, l, static_cast<const float *>(Qw), static_cast<const float *>(K), V, K_out,
+                         V_out, idx_out, s, workspace, st);
+    t_keep_scores = true;
+    return rc;
 }
 
 graphkv_status graphkv_compress_layers(const graphkv_params *params, const int32_t *budgets,
