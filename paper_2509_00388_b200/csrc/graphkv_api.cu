@@ -429,6 +429,7 @@ bool make_k_tensormap(CUtensorMap *tm, const void *K, const Dims &d, int rows, c
 // kernel that follows.
 struct EmitExtras {
     int k;
+    int *list_chunks;   // out: candidate lists per unit the emit sweep leaves (its key chunks)
     int *src_out;
     uint32_t *zero;
     int zero_words;
@@ -464,13 +465,14 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
         tc::ScoreTcArgs sa{d, Q, at<float>(ws, l.part), at<float>(ws, l.row_c), at<int>(ws, l.arrivals), a,
                            ex.global_hist ? at<uint32_t>(ws, l.a_hist) : nullptr, at<int>(ws, l.status), u0,
                            chunks_s, tiles_stats, chunks_s, stages, 0,
-                           tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, nullptr}, nullptr, 0, 0,
+                           tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, 0}, nullptr, 0, 0,
                            wait_cycles(), env_int("GRAPHKV_DEBUG_WITHHOLD_COMMIT", 0)};
         tc::ScoreTcArgs ea = sa;
         ea.chunks = chunks_e;
         ea.n_tiles = tiles_emit;
         ea.src = tc::SourceArgs{ex.k, (d.kp - 1) / 2, ex.src_out, at<tc::SrcCand>(ws, l.src_cand),
-                                at<int>(ws, l.src_cnt), l.max_parts, at<int>(ws, l.arrivals2)};
+                                at<int>(ws, l.src_cnt), l.max_parts, chunks_e};
+        if (ex.list_chunks) *ex.list_chunks = chunks_e;
         ea.zero = ex.zero;
         ea.zero_words = ex.zero_words;
         ea.local_hist = ex.k > 0 ? 1 : 0;
@@ -485,7 +487,7 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
     return rc;
 }
 
-constexpr EmitExtras kPlainEmit{0, nullptr, nullptr, 0, true};
+constexpr EmitExtras kPlainEmit{0, nullptr, nullptr, nullptr, 0, true};
 
 inline bool tc_mass(const __nv_bfloat16 *) { return !env_int("GRAPHKV_FORCE_SIMT", 0); }
 inline bool tc_mass(const float *) { return false; }
@@ -568,9 +570,11 @@ template <typename T> struct EdgeOperands {
     const long long *as;
 };
 
+// `merge` (optional): the sources are still candidate lists the emit sweep left; the similarity
+// sweep merges them (tensor-core path, one sweep of at most 64 sources).
 template <typename T>
 graphkv_status run_graph(const Dims &d, const Layout &l, const EdgeOperands<T> &eo, const int *src, void *ws,
-                         cudaStream_t st)
+                         cudaStream_t st, const tc::SourceArgs *merge = nullptr, const float *a_mass = nullptr)
 {
     const SimPlan sp = sim_plan(d, sizeof(T) == 2);
     if (sp.ok) {
@@ -590,7 +594,8 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const EdgeOperands<T> &
             for (int src0 = 0; src0 < d.K_src; src0 += sp.NP) {
                 tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(eo.S), {eo.ss[0], eo.ss[1], eo.ss[2]}, src, at<Cand>(ws, l.cand),
                                  at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
-                                 sp.n_tiles, sp.stages, 0, wait_cycles(), src0, std::min(sp.NP, d.K_src - src0)};
+                                 sp.n_tiles, sp.stages, 0, wait_cycles(), src0, std::min(sp.NP, d.K_src - src0),
+                                 merge ? *merge : tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, 0}, a_mass};
                 sa.wait_prior = next_launch_is_dependent();
                 const dim3 grid(sp.chunks, nu), block(tc::kSimThreads);
                 graphkv_status rc;
@@ -762,16 +767,19 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
     int *src = at<int>(ws, l.src);
     const bool tc_graph = graph && sim_plan(d, sizeof(T) == 2).ok;
     const int halo = (d.kp - 1) / 2;
-    // The tensor-core emit sweep can pick the sources at its tail and the finishing kernel can pool,
-    // which saves the pooling kernel's launch; measured on B200 the serial tail of the unit's last
-    // emit CTA (about 12 us at 32K keys) costs more than that kernel (10 us), so it is off by default.
+    // The tensor-core emit sweep can leave candidate lists for the sources at its tail, the
+    // similarity sweep merge them and the finishing kernel pool, which saves the pooling kernel
+    // (one sweep of at most 64 sources, one launch group, max pooling).  Measured on B200 the
+    // merge in front of every similarity CTA costs what the pooling kernel takes (32K keys: 114
+    // against 112 us per step; 131072 x 4: 1.25 against 1.13 ms), so it is off by default.
     const bool tail_src = tc_mass(Q) && tc_graph && d.K_src <= tc::kSrcMaxK && !d.pool_avg &&
-                          env_int("GRAPHKV_TAIL_SOURCES", 0);
+                          units_per_group(d) >= d.units && env_int("GRAPHKV_TAIL_SOURCES", 0);
     const bool finish_pools = d.kp > 1 && !d.pool_avg && (tail_src || !graph) && finish_plan(d, halo).ok &&
                               cluster_plan(d).ok;
     graphkv_status rc;
+    int list_chunks = 0;
     if (tail_src || !graph) {
-        const EmitExtras ex{tail_src ? d.K_src : 0, src, tail_src ? at<uint32_t>(ws, l.cand_hist) : nullptr,
+        const EmitExtras ex{tail_src ? d.K_src : 0, &list_chunks, src, tail_src ? at<uint32_t>(ws, l.cand_hist) : nullptr,
                             tail_src ? d.K_src * kCandBins : 0, false};
         if ((rc = run_mass(d, l, Q, K, a, ws, st, ex)) != GRAPHKV_OK) return rc;
         if (d.kp > 1 && !finish_pools &&
@@ -791,7 +799,9 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
         // after it start from the scores in `s`; the last pass also selects and gathers
         Dims one = d;
         one.T = 1;
-        if ((rc = run_graph(one, l, eo, src, ws, st)) != GRAPHKV_OK) return rc;
+        const tc::SourceArgs merge1{d.K_src, halo, src, at<tc::SrcCand>(ws, l.src_cand), at<int>(ws, l.src_cnt),
+                                    l.max_parts, list_chunks};
+        if ((rc = run_graph(one, l, eo, src, ws, st, tail_src ? &merge1 : nullptr, a)) != GRAPHKV_OK) return rc;
         if ((rc = run_finish(one, l, (int)sizeof(T), finish_pools ? a : nullptr, s, true, tc_graph, false,
                              nullptr, nullptr, nullptr, nullptr, nullptr, ws, st)) != GRAPHKV_OK)
             return rc;
@@ -800,7 +810,9 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
         return run_finish(one, l, (int)sizeof(T), nullptr, s, false, false, true, K, V, K_out, V_out, idx_out,
                           ws, st);
     }
-    if (graph && (rc = run_graph(d, l, eo, src, ws, st)) != GRAPHKV_OK) return rc;
+    const tc::SourceArgs merge{d.K_src, halo, src, at<tc::SrcCand>(ws, l.src_cand), at<int>(ws, l.src_cnt),
+                               l.max_parts, list_chunks};
+    if (graph && (rc = run_graph(d, l, eo, src, ws, st, tail_src ? &merge : nullptr, a)) != GRAPHKV_OK) return rc;
     return run_finish(d, l, (int)sizeof(T), finish_pools ? a : nullptr, s, graph, tc_graph, true, K, V,
                       K_out, V_out, idx_out, ws, st);
 }

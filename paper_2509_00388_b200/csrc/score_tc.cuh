@@ -47,7 +47,7 @@ struct ScoreTcArgs {
     int stats_chunks;   // key chunks of the statistics sweep (partials per row)
     int stages;         // shared-memory K tiles in flight
     int wait_prior;     // launched with programmatic stream serialization: wait for the kernels before
-    // emit sweep only: the source nodes of Eq. 2 at its tail (src.k = 0: none), and words to clear
+    // emit sweep only: candidate lists for the source nodes of Eq. 2 at its tail (src.k = 0: none), and words to clear
     // for the kernels that follow
     SourceArgs src;
     uint32_t *zero;     // optional [units][zero_words]
@@ -529,10 +529,11 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads)
             if (mass_hist[i]) atomicAdd(a.a_hist + (long long)unit * kMassBins + i, mass_hist[i]);
     pc.mark();
-    // Eq. 2: the unit's source nodes (the stage ring is idle by now and serves as scratch)
+    // Eq. 2, first half: this chunk's candidates for the unit's source nodes (the stage ring is idle
+    // by now and serves as scratch); the similarity sweep merges the lists
     if (a.src.k > 0 && all_ok)
-        source_select_tail(a.src, d, unit, chunk, a.chunks, t0 * kTileKeys, min(t1 * kTileKeys, d.N),
-                           a.a_out + (long long)unit * d.N, mass_hist, gen + (s.stage0 - s.q));
+        source_list_chunk(a.src, d, unit, chunk, t0 * kTileKeys, min(t1 * kTileKeys, d.N),
+                          a.a_out + (long long)unit * d.N, mass_hist, gen + (s.stage0 - s.q));
     pc.mark();
     pc.flush(1);
 }

@@ -20,6 +20,7 @@
 // takes a bound that leaves it a few dozen edges to rank.
 #pragma once
 
+#include "source_select.cuh"
 #include "tc_common.cuh"
 
 namespace graphkv {
@@ -47,6 +48,9 @@ struct SimTcArgs {
     int wait_prior;        // launched with programmatic stream serialization
     long long wait_cycles; // limit of every wait of the kernel, in clocks
     int src0, n_src;       // this launch takes sources [src0, src0 + n_src) of every unit (n_src <= NP)
+    SourceArgs merge;      // merge.k > 0: the sources are not in `src` yet; every CTA merges the candidate
+                           // lists the emit sweep left (Eq. 2) and the first chunk of a unit writes them to `src`
+    const float *a_mass;   // [units][N] attention mass the merge pools (merge.k > 0)
 };
 
 template <int NP> __host__ __device__ constexpr int sim_tiles_cap() { return 512 / NP; }
@@ -133,7 +137,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         tma_prefetch_desc(&tmK);
         // the first ring-full of key tiles is under way while the sources are gathered (keys are an
         // input of the call: no wait for the kernels before)
-        n_ahead = min(a.stages, n_local);
+        // (a merge of candidate lists borrows the last two stages as scratch first)
+        n_ahead = min(a.merge.k > 0 ? a.stages - 2 : a.stages, n_local);
         for (int i = 0; i < n_ahead; ++i) {
             const uint32_t dst = s_stage0 + i * kTileBytes;
             mbar_expect_tx(s_full0 + 8 * i, kTileBytes);
@@ -149,6 +154,12 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     if (a.wait_prior) pdl_wait();
     pdl_launch_dependents();
     pc.mark();
+    if (a.merge.k > 0) {
+        static_assert(2 * kTileBytes >= kSrcSmemBytes, "the merge's scratch fits two stages");
+        source_merge(a.merge, d, unit, a.a_mass + (long long)unit * d.N,
+                     gen + (s_stage0 - base) + (a.stages - 2) * kTileBytes, src_pos,
+                     chunk == 0 ? const_cast<int *>(src) : nullptr);
+    }
     // source keys -> swizzled operand rows (rows >= K_src are zero), their positions and norms
     // (16 consecutive threads share a row: the row's squared norm is reduced among them)
     for (int i0 = 0; i0 < NP * 16; i0 += kSimThreads) {
@@ -158,7 +169,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         uint4 v = make_uint4(0, 0, 0, 0);
         int pos = -1;
         if (in && r < n_src) {
-            pos = src[r];
+            pos = a.merge.k > 0 ? src_pos[r] : src[r];
             v = *reinterpret_cast<const uint4 *>(Sh + (long long)pos * a.ss[2] + c16 * 8);
         }
         if (in) *reinterpret_cast<uint4 *>(gen + sw128_offset(NP, r, c16)) = v;

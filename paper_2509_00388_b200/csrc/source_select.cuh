@@ -1,16 +1,17 @@
-// Eq. 2 at the tail of the emit sweep: the source nodes of a unit, the top-k of the POOLED scores
-// s_j = max(a[j - h .. j + h]), found without another kernel and without pooling the whole row.
+// Eq. 2 without a kernel of its own: the source nodes of a unit, the top-k of the POOLED scores
+// s_j = max(a[j - h .. j + h]), found without pooling the whole row.
 //
-// Every CTA of the emit sweep lists the elements of its key chunk whose attention mass reaches the
-// chunk's own k-th largest (first by the chunk's mass histogram, then exactly among those: k of
-// them plus ties).  The CTA of a unit that finishes last merges the lists.  Let v be
-// the k-th largest mass of the unit (it is among the listed: an element that k others of its own
-// chunk exceed cannot be it).  Pooling only raises values, so k positions have s >= v and every
-// source has s_j >= v; such a position lies within h of an element with a >= v.  The elements with
-// a >= v (k of them plus ties) are all listed, so the merge pools exactly the positions within h
-// of them, ranks those (score descending, position ascending) and keeps k.  Rows with massive
-// ties (more than kSrcPeaks elements at or above v, or a chunk list that outgrew its slots) take
-// a plain radix search over the pooled row instead, by the same CTA: rare, and slow.
+// Every CTA of the emit sweep lists, at its tail, the elements of its key chunk whose attention
+// mass reaches the chunk's own k-th largest (first by the chunk's mass histogram, then exactly
+// among those: k of them plus ties).  Every CTA of the similarity sweep that follows merges the
+// lists of its unit for itself, before it gathers the source keys.  Let v be the k-th largest
+// mass of the unit (it is among the listed: an element that k others of its own chunk exceed
+// cannot be it).  Pooling only raises values, so k positions have s >= v and every source has
+// s_j >= v; such a position lies within h of an element with a >= v.  The elements with a >= v
+// (k of them plus ties) are all listed, so the merge pools exactly the positions within h of
+// them, ranks those (score descending, position ascending) and keeps k.  Rows with massive ties
+// (more than kSrcPeaks elements at or above v, or a chunk list that outgrew its slots) take a
+// plain radix search over the pooled row instead: rare, and slow.
 #pragma once
 
 #include "common.cuh"
@@ -36,7 +37,7 @@ struct SourceArgs {
     SrcCand *cand;          // [units][chunk_slots][kSrcCap] listed elements per chunk
     int *cand_n;            // [units][chunk_slots] their number (kSrcCap + 1: the list overflowed)
     int chunk_slots;
-    int *arrivals;          // [units] emit CTAs done per unit (zero before the launch; reset on the way)
+    int chunks;             // lists per unit (the key chunks of the emit sweep)
 };
 
 // Shared memory the tail needs, in bytes (it reuses the stage ring of the sweep, idle by then).
@@ -123,18 +124,17 @@ __device__ void source_select_general(const float *a_row, int N, int h, int k, i
 }
 
 // Called by all threads of an emit CTA after its tile loop (the chunk's mass values are in global
-// memory, its mass histogram in `mass_hist`).  `scratch`: kSrcSmemBytes of shared memory.
-__device__ void source_select_tail(const SourceArgs &sa, const Dims &d, int unit, int chunk,
-                                   int chunks, int j_begin, int j_end, const float *a_row,
-                                   const uint32_t *mass_hist, uint8_t *scratch)
+// memory, its mass histogram in `mass_hist`): lists the chunk's candidates for the merge.
+// `scratch`: kSrcSmemBytes of shared memory.
+__device__ void source_list_chunk(const SourceArgs &sa, const Dims &d, int unit, int chunk,
+                                  int j_begin, int j_end, const float *a_row,
+                                  const uint32_t *mass_hist, uint8_t *scratch)
 {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
-    const int k = sa.k, h = sa.halo, N = d.N;
+    const int k = sa.k;
+    (void)d;
     SrcCand *merged = reinterpret_cast<SrcCand *>(scratch);                    // [kSrcMerge]
-    int *peaks = reinterpret_cast<int *>(merged + kSrcMerge);                  // [kSrcPeaks]
-    SrcCand *pool = reinterpret_cast<SrcCand *>(peaks + kSrcPeaks);            // [kSrcPool]
-    uint32_t *hist = reinterpret_cast<uint32_t *>(pool + kSrcPool);            // [2048]
-    uint32_t *misc = hist + 2048;                                              // [64]
+    uint32_t *misc = reinterpret_cast<uint32_t *>(merged + kSrcMerge);         // [64]
     // 1. the chunk's threshold bin: the highest bin with k of its elements in or above it
     if (tid == 0) {
         misc[0] = 0u;
@@ -206,16 +206,23 @@ __device__ void source_select_tail(const SourceArgs &sa, const Dims &d, int unit
         for (int i = tid; i < min(n_mine, kSrcCap); i += nthr) sa.cand[slot0 * kSrcCap + i] = mine[i];
     }
     if (tid == 0) sa.cand_n[slot0] = n_mine > kSrcCap ? kSrcCap + 1 : n_mine;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) misc[2] = atomicAdd(sa.arrivals + unit, 1) == chunks - 1 ? 1u : 0u;
-    __syncthreads();
-    if (!misc[2]) return;
-    // ---- the unit's last CTA: merge ----
-    __threadfence();
-    int *src_out = sa.src_out + (long long)unit * k;
+}
+
+// Called by all threads of a CTA (at least kSrcPeaks of them) once every list of the unit is
+// complete: the unit's k sources by ascending position into `out` (shared memory) and, when
+// `out_global` is given, into global memory too.  `scratch`: kSrcSmemBytes of shared memory.
+// Ends with the CTA synchronised.
+__device__ void source_merge(const SourceArgs &sa, const Dims &d, int unit, const float *a_row,
+                             uint8_t *scratch, int *out, int *out_global)
+{
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int k = sa.k, h = sa.halo, N = d.N, chunks = sa.chunks;
+    SrcCand *merged = reinterpret_cast<SrcCand *>(scratch);                    // [kSrcMerge]
+    int *peaks = reinterpret_cast<int *>(merged + kSrcMerge);                  // [kSrcPeaks]
+    SrcCand *pool = reinterpret_cast<SrcCand *>(peaks + kSrcPeaks);            // [kSrcPool]
+    uint32_t *hist = reinterpret_cast<uint32_t *>(pool + kSrcPool);            // [2048]
+    uint32_t *misc = hist + 2048;                                              // [64]
     if (tid == 0) {
-        sa.arrivals[unit] = 0;                              // ready for the next launch
         misc[3] = 0u;                                       // merged elements
         misc[4] = 0u;                                       // 1: take the general path
         misc[5] = 0u;                                       // peaks
@@ -302,13 +309,19 @@ __device__ void source_select_tail(const SourceArgs &sa, const Dims &d, int unit
                 const int p = kept[tid];
                 int o = 0;
                 for (int u = 0; u < k; ++u) o += kept[u] < p;
-                src_out[o] = p;
+                out[o] = p;
+                if (out_global) out_global[o] = p;
             }
+            __syncthreads();
             return;
         }
     }
     __syncthreads();
-    source_select_general(a_row, N, h, k, src_out, hist, reinterpret_cast<int *>(merged), misc);
+    source_select_general(a_row, N, h, k, out, hist, reinterpret_cast<int *>(merged), misc);
+    __syncthreads();
+    if (out_global)
+        for (int i = tid; i < k; i += nthr) out_global[i] = out[i];
+    __syncthreads();
 }
 
 }  // namespace tc
