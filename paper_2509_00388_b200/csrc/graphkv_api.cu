@@ -29,7 +29,6 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t status;      // int status word (256 bytes reserved)
     size_t arrivals;    // stats CTAs done per unit [units] (directly after the status word)
-    size_t arrivals2;   // emit CTAs done per unit [units] (directly after those)
     size_t a_hist;      // histogram of the attention mass [units][2048] (directly after the counters)
     size_t row_c;       // softmax row constants [units][GW]
     size_t part;        // softmax row statistics per key chunk
@@ -211,7 +210,6 @@ Layout layout_of(const Dims &d)
     l.max_parts = l.n_stat_chunks > 148 ? l.n_stat_chunks : 148;
     l.status = take(kAlign);
     l.arrivals = take((size_t)d.units * sizeof(int));
-    l.arrivals2 = take((size_t)d.units * sizeof(int));
     l.a_hist = take((size_t)d.units * tc::kMassBins * sizeof(uint32_t));
     l.row_c = take((size_t)d.units * d.GW * sizeof(float));
     l.part = take((size_t)d.units * l.max_parts * d.GW * 2 * sizeof(float));
@@ -819,34 +817,33 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
 
 // ---- KNorm initial score ---------------------------------------------------------------------
 // s_j = 1 / max(||k_j||, eps) for the prefix keys: 16 threads share a key row (16 bytes each of a
-// bf16 row, 32 of an fp32 row), four rows in flight per thread.  grid-stride over units * N rows.
+// bf16 row, 32 of an fp32 row), eight rows in flight per thread.  grid (CTAs per unit, units).
 template <typename T>
 __global__ void __launch_bounds__(256) knorm_score_kernel(Dims d, const T *__restrict__ K, float *__restrict__ scores)
 {
-    const int sub = threadIdx.x & 15;
-    const long long rows = (long long)d.units * d.N;
-    const long long stride = ((long long)gridDim.x * blockDim.x) >> 4;
-    for (long long r0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 4; r0 < rows; r0 += 4 * stride) {
-        float n2[4];
+    const int sub = threadIdx.x & 15, unit = blockIdx.y;
+    const T *Kh = K + (unit / d.hkv) * d.ks[0] + (long long)(unit % d.hkv) * d.ks[1] + sub * (kHeadDim / 16);
+    float *out = scores + (long long)unit * d.N;
+    const int stride = (gridDim.x * blockDim.x) >> 4;
+    for (int j0 = (blockIdx.x * blockDim.x + threadIdx.x) >> 4; j0 < d.N; j0 += 8 * stride) {
+        float n2[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const long long r = r0 + u * stride;
+        for (int u = 0; u < 8; ++u) {
+            const int j = j0 + u * stride;
             n2[u] = 0.f;
-            if (r < rows) {
-                const int unit = (int)(r / d.N), j = (int)(r % d.N);
-                const T *row = K + (unit / d.hkv) * d.ks[0] + (long long)(unit % d.hkv) * d.ks[1] + (long long)j * d.ks[2];
+            if (j < d.N) {
                 float v[8];
-                load8(row + sub * 8, v);
+                load8(Kh + (long long)j * d.ks[2], v);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) n2[u] = fmaf(v[e], v[e], n2[u]);
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) n2[u] += __shfl_xor_sync(0xffffffffu, n2[u], o);
-            const long long r = r0 + u * stride;
-            if (sub == 0 && r < rows) scores[r] = 1.0f / fmaxf(sqrtf(n2[u]), kNormEps);
+            const int j = j0 + u * stride;
+            if (sub == 0 && j < d.N) out[j] = 1.0f / fmaxf(sqrtf(n2[u]), kNormEps);
         }
     }
 }
@@ -988,14 +985,14 @@ graphkv_status graphkv_score_knorm(const graphkv_params *params, const void *K, 
     if (rc != GRAPHKV_OK) return rc;
     if (!K || !scores || !aligned16(K)) return GRAPHKV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const long long rows = (long long)d.units * d.N;
-    // one wave of resident CTAs (eight of 256 threads per SM), each group of 16 threads taking rows in steps
-    const int blocks = (int)std::min<long long>((rows * 16 + 255) / 256, (long long)sm_count() * 8);
+    // about one wave of resident CTAs (eight of 256 threads per SM) over all units
+    const int per_unit = std::max(1, std::min(ceil_div(d.N, 16 * 8), ceil_div(sm_count() * 8, d.units)));
+    const dim3 grid(per_unit, d.units);
     if (params->dtype == GRAPHKV_BF16)
-        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
                                           d, static_cast<const __nv_bfloat16 *>(K), scores)));
     else
-        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<float><<<blocks, 256, 0, st>>>(
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<float><<<grid, 256, 0, st>>>(
                                           d, static_cast<const float *>(K), scores)));
     return launch_status();
 }

@@ -104,3 +104,32 @@ def test_binding_has_no_cpu_route():
     import inspect
     src = inspect.getsource(gk)
     assert "oracle" not in src
+
+
+def test_variant_fields_and_entry_points_validate_on_the_host():
+    lib = gk.lib()
+    for bad in (dict(signal=3), dict(signal=-1), dict(reselect=2), dict(pool_mode=2)):
+        assert gk.workspace_bytes(_params(**bad)) == 0
+    for ok in (dict(signal=gk.SIGNAL_EVICT), dict(reselect=1), dict(pool_mode=gk.POOL_AVG)):
+        assert gk.workspace_bytes(_params(**ok)) > 0
+    p = _params()
+    # edge operands: unknown tensor kind, missing tensor
+    assert lib.graphkv_propagate_edges(C.byref(p), 256, None, 0, 7, 256, None, 256, 1 << 30, None) == gk.ERR_INVALID_ARG
+    assert lib.graphkv_propagate_edges(C.byref(p), 256, None, gk.TENSOR_V, gk.TENSOR_V, 256, None, 256, 1 << 30,
+                                       None) == gk.ERR_INVALID_ARG
+    assert lib.graphkv_score_knorm(C.byref(p), None, 256, None) == gk.ERR_INVALID_ARG
+    # per-layer budgets: each within 1 .. params.budget, at most 64 layers
+    arr = (C.c_int32 * 1)(11)
+    assert lib.graphkv_compress_layers(C.byref(p), arr, 256, 256, 256, 256, 256, 256, None, 256, 1 << 30,
+                                       None) == gk.ERR_INVALID_ARG
+    assert lib.graphkv_compress_layers(C.byref(p), None, 256, 256, 256, 256, 256, 256, None, 256, 1 << 30,
+                                       None) == gk.ERR_INVALID_ARG
+    # decode attention: shape checks and workspace sizing without a device
+    q = torch.empty(1, 4, 128, dtype=torch.bfloat16)
+    K = torch.empty(1, 2, 100, 128, dtype=torch.bfloat16)
+    dp = gk.decode_params(q, K, K)
+    need = int(lib.graphkv_decode_workspace_bytes(C.byref(dp)))
+    assert need > 0 and need % 256 == 0
+    assert lib.graphkv_decode_attention(C.byref(dp), 256, 256, 256, 256, 256, need - 1, None) == gk.ERR_WORKSPACE
+    q9 = torch.empty(1, 18, 128, dtype=torch.bfloat16)       # 9 query heads per KV head: beyond the kernel
+    assert int(lib.graphkv_decode_workspace_bytes(C.byref(gk.decode_params(q9, K, K)))) == 0
