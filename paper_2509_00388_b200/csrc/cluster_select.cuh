@@ -50,13 +50,13 @@ struct Smem {
     float *st_f;          // [kStage] staging: decay factors / survivors
     int *nb_j;            // [stage_cap] the unit's neighbour lists, positions (every CTA holds a copy)
     float *nb_f;          // [stage_cap] their decay factors over all rounds
-    int stage_cap;        // words of each of the four staging arrays (at least kStage)
+    int stage_cap;        // words of nb_j and of nb_f (at least kStage)
     float *vals;          // [halo + chunk + halo]
 };
 
 __host__ __device__ inline size_t smem_bytes(int chunk, int halo, int stage_cap = kStage)
 {
-    return (size_t)(kBins + kTotWords + kFineBins + 2 * kWarps + 32 + 4 * stage_cap) * 4 +
+    return (size_t)(kBins + kTotWords + kFineBins + 2 * kWarps + 32 + 2 * kStage + 2 * stage_cap) * 4 +
            (size_t)(chunk + 2 * halo + 8) * 4;
 }
 
@@ -69,8 +69,8 @@ __device__ __forceinline__ Smem carve(uint8_t *raw, int halo, int stage_cap = kS
     s.wcnt = s.fine + kFineBins;
     s.misc = s.wcnt + 2 * kWarps;
     s.st_idx = reinterpret_cast<int *>(s.misc + 32);
-    s.st_f = reinterpret_cast<float *>(s.st_idx + stage_cap);
-    s.nb_j = reinterpret_cast<int *>(s.st_f + stage_cap);
+    s.st_f = reinterpret_cast<float *>(s.st_idx + kStage);
+    s.nb_j = reinterpret_cast<int *>(s.st_f + kStage);
     s.nb_f = reinterpret_cast<float *>(s.nb_j + stage_cap);
     s.vals = s.nb_f + stage_cap;
     s.stage_cap = stage_cap;
@@ -1082,6 +1082,30 @@ __device__ void apply_lists(const Smem &s, float *vals, int base, int n_local, i
 {
     const int tid = threadIdx.x;
     const int pairs = K_src * m;                           // fits the staging arrays
+    if (pairs > kStage) {
+        // hundreds of sources, whose neighbourhoods overlap heavily (counting the edges per position
+        // would serialise on the few positions they share): one warp applies the lists source
+        // after source, the next source's entries read ahead
+        if (tid < 32) {
+            int jn = tid < m ? s.nb_j[tid] - base : -1;
+            float fn = tid < m ? s.nb_f[tid] : 1.f;
+            for (int q = 0; q < K_src; ++q) {
+                for (int u = tid; u < m; u += 32) {
+                    const bool first = u == tid;
+                    const int j = first ? jn : s.nb_j[q * m + u] - base;
+                    const float f = first ? fn : s.nb_f[q * m + u];
+                    if (j >= 0 && j < n_local) vals[j] = evict ? -INFINITY : vals[j] * f;
+                }
+                if (q + 1 < K_src && tid < m) {
+                    jn = s.nb_j[(q + 1) * m + tid] - base;
+                    fn = s.nb_f[(q + 1) * m + tid];
+                }
+                __syncwarp();
+            }
+        }
+        __syncthreads();
+        return;
+    }
     uint32_t *cnt = s.fine;                                // [4096] edges per table slot
     uint32_t *src_mask = s.fine + 4096;                    // [K_src / 32] sources with a contested edge
     for (int i = tid; i < 4096 + (K_src + 31) / 32; i += kThreads) cnt[i] = 0u;
