@@ -589,25 +589,24 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const EdgeOperands<T> &
         const int group = units_per_group(d);
         for (int u0 = 0; u0 < d.units; u0 += group) {
             const int nu = std::min(group, d.units - u0);
-            for (int src0 = 0; src0 < d.K_src; src0 += sp.NP) {
-                tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(eo.S), {eo.ss[0], eo.ss[1], eo.ss[2]}, src, at<Cand>(ws, l.cand),
-                                 at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
-                                 sp.n_tiles, sp.stages, 0, wait_cycles(), src0, std::min(sp.NP, d.K_src - src0),
-                                 merge ? *merge : tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, 0}, a_mass};
-                sa.wait_prior = next_launch_is_dependent();
-                const dim3 grid(sp.chunks, nu), block(tc::kSimThreads);
-                graphkv_status rc;
-                if (sp.NP == 16)
-                    rc = launch_ex("similarity_tc", tc::similarity_tc<16>, grid, block,
-                                   tc::sim_smem_bytes<16>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
-                else if (sp.NP == 32)
-                    rc = launch_ex("similarity_tc", tc::similarity_tc<32>, grid, block,
-                                   tc::sim_smem_bytes<32>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
-                else
-                    rc = launch_ex("similarity_tc", tc::similarity_tc<64>, grid, block,
-                                   tc::sim_smem_bytes<64>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
-                if (rc != GRAPHKV_OK) return rc;
-            }
+            // one launch takes every source: grid.z counts the sweeps of sp.NP sources each
+            tc::SimTcArgs sa{d, reinterpret_cast<const __nv_bfloat16 *>(eo.S), {eo.ss[0], eo.ss[1], eo.ss[2]}, src, at<Cand>(ws, l.cand),
+                             at<uint32_t>(ws, l.cand_hist), at<int>(ws, l.status), u0, sp.chunks,
+                             sp.n_tiles, sp.stages, 0, wait_cycles(),
+                             merge ? *merge : tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, 0}, a_mass};
+            sa.wait_prior = next_launch_is_dependent();
+            const dim3 grid(sp.chunks, nu, ceil_div(d.K_src, sp.NP)), block(tc::kSimThreads);
+            graphkv_status rc;
+            if (sp.NP == 16)
+                rc = launch_ex("similarity_tc", tc::similarity_tc<16>, grid, block,
+                               tc::sim_smem_bytes<16>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
+            else if (sp.NP == 32)
+                rc = launch_ex("similarity_tc", tc::similarity_tc<32>, grid, block,
+                               tc::sim_smem_bytes<32>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
+            else
+                rc = launch_ex("similarity_tc", tc::similarity_tc<64>, grid, block,
+                               tc::sim_smem_bytes<64>(sp.stages), st, sa.wait_prior != 0, 1, tmK, sa);
+            if (rc != GRAPHKV_OK) return rc;
         }
         return GRAPHKV_OK;
     }

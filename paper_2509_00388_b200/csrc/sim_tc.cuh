@@ -3,7 +3,7 @@
 // source's top-m neighbourhood (Eq. 3).  The edge matrix never leaves the SM.
 //
 // One CTA owns a chunk of at most 512 / NP key tiles of one head (NP = source count padded to
-// 16, 32 or 64; a head with more sources is swept once per 64 of them).  Each 128-key tile arrives by TMA, one tcgen05.mma block computes its
+// 16, 32 or 64; a head with more sources is swept once per 64 of them, by CTAs of their own).  Each 128-key tile arrives by TMA, one tcgen05.mma block computes its
 // 128 x NP dot products against the source keys into its own TMEM columns, and the epilogue
 // threads (thread = key) take the key's norm from the staged tile.  When the sweep is over the
 // chunk's whole edge block still sits in TMEM, and the CTA
@@ -47,7 +47,6 @@ struct SimTcArgs {
     int stages;
     int wait_prior;        // launched with programmatic stream serialization
     long long wait_cycles; // limit of every wait of the kernel, in clocks
-    int src0, n_src;       // this launch takes sources [src0, src0 + n_src) of every unit (n_src <= NP)
     SourceArgs merge;      // merge.k > 0: the sources are not in `src` yet; every CTA merges the candidate
                            // lists the emit sweep left (Eq. 2) and the first chunk of a unit writes them to `src`
     const float *a_mass;   // [units][N] attention mass the merge pools (merge.k > 0)
@@ -123,8 +122,10 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     const int t0 = chunk * per + min(chunk, rem);
     const int n_local = per + (chunk < rem ? 1 : 0);
     const __nv_bfloat16 *Sh = a.S + b * a.ss[0] + (long long)h * a.ss[1];
-    const int *src = a.src + (long long)unit * d.K_src + a.src0;
-    const int n_src = a.n_src;                               // sources of this launch
+    // a head with more than NP sources is swept once per NP of them: grid.z counts those sweeps
+    const int src0 = blockIdx.z * NP;
+    const int *src = a.src + (long long)unit * d.K_src + src0;
+    const int n_src = min(NP, d.K_src - src0);               // sources of this CTA
 
     int n_ahead = 0;                 // tiles thread 0 has requested before the roles split
     if (threadIdx.x == 0) {
@@ -446,18 +447,18 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             // write the lists out (unused slots marked empty) and count the listed edges per bin
             for (int idx = et; idx < n_src * kCandCap; idx += kSimEpiThreads) {
                 const int c = idx / kCandCap, q = idx % kCandCap;
-                const long long slot = ((long long)unit * d.K_src + a.src0 + c) * a.chunks + chunk;
+                const long long slot = ((long long)unit * d.K_src + src0 + c) * a.chunks + chunk;
                 Cand cd{kCandEmpty, -1};
                 if (q < min(cnt[c], kCandCap)) {
                     cd = list[c * kCandCap + q];
-                    atomicAdd(a.cand_hist + ((long long)unit * d.K_src + a.src0 + c) * kCandBins + cand_bin(cd.e), 1u);
+                    atomicAdd(a.cand_hist + ((long long)unit * d.K_src + src0 + c) * kCandBins + cand_bin(cd.e), 1u);
                 }
                 a.cand[slot * kCandCap + q] = cd;
             }
         } else {
             // a wait ran out: publish empty lists so the merge reads nothing undefined
             for (int i = et; i < n_src * kCandCap; i += kSimEpiThreads) {
-                const long long slot = ((long long)unit * d.K_src + a.src0 + i / kCandCap) * a.chunks + chunk;
+                const long long slot = ((long long)unit * d.K_src + src0 + i / kCandCap) * a.chunks + chunk;
                 a.cand[slot * kCandCap + i % kCandCap] = Cand{kCandEmpty, -1};
             }
         }
