@@ -626,12 +626,20 @@ __device__ void merge_neighbours(cg::cluster_group &cl, const Cand *cand, const 
     const int lane = threadIdx.x & 31;
     constexpr int kPer = kCandBins / 32;
     // lane l holds bins [l * kPer, (l + 1) * kPer); walk down from the top bin
+    // the histogram and the group's first block of 256 slots per warp are requested together: one
+    // round trip to memory instead of two
+    const int slots = chunks * kCandCap;
     uint32_t h[kPer], mine = 0;
+    unsigned long long raw[8];
 #pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-        h[q] = __ldcg(hist + lane * kPer + q);
-        mine += h[q];
+    for (int q = 0; q < kPer; ++q) h[q] = __ldcg(hist + lane * kPer + q);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int i = wg * 256 + q * 32 + lane;
+        raw[q] = i < slots ? __ldcg(reinterpret_cast<const unsigned long long *>(cand + i)) : 0ull;
     }
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) mine += h[q];
     uint32_t above = 0;                       // listed edges in the lanes above this one
     {
         uint32_t incl = mine;              // suffix sum over lanes, log steps
@@ -654,30 +662,37 @@ __device__ void merge_neighbours(cg::cluster_group &cl, const Cand *cand, const 
     for (int o = 16; o > 0; o >>= 1) bstar = max(bstar, __shfl_xor_sync(0xffffffffu, bstar, o));
     const float bound = bstar <= 0 ? -1.0f : (float)bstar / (float)kCandBins;
 
-    // the four warps of the group take interleaved blocks of 256 slots, eight loads in flight per lane
+    // the four warps of the group take interleaved blocks of 256 slots; a warp reserves the places
+    // of a block's survivors with one addition
     if (wg == 0 && lane == 0) *ns_sh = 0;
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-    const int slots = chunks * kCandCap;
     for (int i0 = wg * 256; i0 < slots; i0 += 4 * 256) {
-        unsigned long long raw[8];
+        if (i0 != wg * 256) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int i = i0 + q * 32 + lane;
-            raw[q] = i < slots ? __ldcg(reinterpret_cast<const unsigned long long *>(cand + i)) : 0ull;
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int i = i0 + q * 32 + lane;
-            const Cand cd{__uint_as_float(static_cast<uint32_t>(raw[q])), static_cast<int>(raw[q] >> 32)};
-            const bool keep = i < slots && cd.e >= bound;
-            const unsigned bm = __ballot_sync(0xffffffffu, keep);
-            if (bm) {
-                int basep = 0;
-                if (lane == 0) basep = atomicAdd(ns_sh, __popc(bm));
-                basep = __shfl_sync(0xffffffffu, basep, 0);
-                const int pos = basep + __popc(bm & ((1u << lane) - 1u));
-                if (keep && pos < kSurvCap) surv[pos] = cd;
+            for (int q = 0; q < 8; ++q) {
+                const int i = i0 + q * 32 + lane;
+                raw[q] = i < slots ? __ldcg(reinterpret_cast<const unsigned long long *>(cand + i)) : 0ull;
             }
+        }
+        unsigned bm[8];
+        int total = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = i0 + q * 32 + lane;
+            const float e = __uint_as_float(static_cast<uint32_t>(raw[q]));
+            bm[q] = __ballot_sync(0xffffffffu, i < slots && e >= bound);
+            total += __popc(bm[q]);
+        }
+        if (total == 0) continue;
+        int basep = 0;
+        if (lane == 0) basep = atomicAdd(ns_sh, total);
+        basep = __shfl_sync(0xffffffffu, basep, 0);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int pos = basep + __popc(bm[q] & ((1u << lane) - 1u));
+            if (((bm[q] >> lane) & 1u) && pos < kSurvCap)
+                surv[pos] = Cand{__uint_as_float(static_cast<uint32_t>(raw[q])), static_cast<int>(raw[q] >> 32)};
+            basep += __popc(bm[q]);
         }
     }
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
@@ -1084,23 +1099,34 @@ __device__ void apply_lists(const Smem &s, float *vals, int base, int n_local, i
     const int pairs = K_src * m;                           // fits the staging arrays
     if (pairs > kStage) {
         // hundreds of sources, whose neighbourhoods overlap heavily (counting the edges per position
-        // would serialise on the few positions they share): one warp applies the lists source
-        // after source, the next source's entries read ahead
-        if (tid < 32) {
-            int jn = tid < m ? s.nb_j[tid] - base : -1;
-            float fn = tid < m ? s.nb_f[tid] : 1.f;
-            for (int q = 0; q < K_src; ++q) {
-                for (int u = tid; u < m; u += 32) {
-                    const bool first = u == tid;
-                    const int j = first ? jn : s.nb_j[q * m + u] - base;
-                    const float f = first ? fn : s.nb_f[q * m + u];
-                    if (j >= 0 && j < n_local) vals[j] = evict ? -INFINITY : vals[j] * f;
+        // would serialise on the few positions they share): every warp walks the whole list, 32
+        // entries at a time, and applies the entries of the positions it owns (a position belongs to
+        // one warp, so its factors are applied in list order, whatever the other warps do)
+        const int warp = tid >> 5, lane = tid & 31;
+        for (int i0 = 0; i0 < pairs; i0 += 32) {
+            const int i = i0 + lane;
+            int j = -1;
+            float f = 1.f;
+            if (i < pairs) {
+                j = s.nb_j[i] - base;
+                f = s.nb_f[i];
+            }
+            const bool own = j >= 0 && j < n_local && ((j >> 2) & 31) == warp;
+            const unsigned ob = __ballot_sync(0xffffffffu, own);
+            if (ob == 0) continue;
+            if ((ob & (ob - 1)) == 0) {                       // one entry: no order to keep
+                if (own) vals[j] = evict ? -INFINITY : vals[j] * f;
+                continue;
+            }
+            if (own) {
+                // lanes that hold the same position take turns, lowest lane first
+                const unsigned peers = __match_any_sync(ob, j);
+                unsigned todo = peers;
+                while (todo) {
+                    if (__ffs(todo) - 1 == lane) vals[j] = evict ? -INFINITY : vals[j] * f;
+                    todo &= todo - 1;
+                    __syncwarp(peers);
                 }
-                if (q + 1 < K_src && tid < m) {
-                    jn = s.nb_j[(q + 1) * m + tid] - base;
-                    fn = s.nb_f[(q + 1) * m + tid];
-                }
-                __syncwarp();
             }
         }
         __syncthreads();

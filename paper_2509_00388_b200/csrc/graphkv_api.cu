@@ -170,6 +170,11 @@ ClusterPlan cluster_plan(const Dims &d)
     // wave of clusters of 4 for 32 rows of 131072)
     while (p.C < cs::kMaxCluster && ceil_div(d.N, p.C) > 4096) p.C *= 2;
     while (p.C > 1 && d.units * p.C > sm_count() && ceil_div(d.N, p.C / 2) <= cs::kMaxChunk) p.C /= 2;
+    // hundreds of sources: their neighbour lists are merged by groups of warps, kMergeWarps per CTA,
+    // so more CTAs per row shorten that phase as long as all clusters stay in one wave
+    while (d.K_src > 4 * cs::kMergeWarps * p.C && p.C < cs::kMaxCluster && d.units * p.C * 2 <= sm_count() &&
+           ceil_div(d.N, p.C * 2) >= 1024)
+        p.C *= 2;
     p.chunk = (ceil_div(d.N, p.C) + 31) & ~31;
     p.ok = p.chunk <= cs::kMaxChunk && p.halo <= cs::kMaxHalo;
     return p;
