@@ -80,6 +80,7 @@ def algorithmic_bytes(cfg, kernel: str) -> float:
     q_bytes = cfg.batch * cfg.n_q_heads * W * D * e
     row = 4 * units * N
     table = {
+        "score_fused": k_sweep + q_bytes + row,
         "score_stats": k_sweep + q_bytes,
         "score_emit": units * N * D * e + q_bytes + row,
         "pool_max": 2 * row,

@@ -28,7 +28,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Workspace carve-up; every region starts 256-byte aligned.
 struct Layout {
     size_t status;      // int status word (256 bytes reserved)
-    size_t arrivals;    // stats CTAs done per unit [units] (directly after the status word)
+    size_t arrivals;    // counters of score CTAs per unit [2 * units] (directly after the status word)
     size_t a_hist;      // histogram of the attention mass [units][2048] (directly after the counters)
     size_t row_c;       // softmax row constants [units][GW]
     size_t part;        // softmax row statistics per key chunk
@@ -214,7 +214,7 @@ Layout layout_of(const Dims &d)
     l.n_stat_chunks = ceil_div(d.L, kStatsChunk);
     l.max_parts = l.n_stat_chunks > 148 ? l.n_stat_chunks : 148;
     l.status = take(kAlign);
-    l.arrivals = take((size_t)d.units * sizeof(int));
+    l.arrivals = take((size_t)d.units * 2 * sizeof(int));
     l.a_hist = take((size_t)d.units * tc::kMassBins * sizeof(uint32_t));
     l.row_c = take((size_t)d.units * d.GW * sizeof(float));
     l.part = take((size_t)d.units * l.max_parts * d.GW * 2 * sizeof(float));
@@ -455,7 +455,8 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
     if (!once_per_device(mu, state, [] {
         const size_t mx = std::max(tc::score_smem_bytes(256, 4), tc::score_smem_bytes(128, 5));
         return set_smem(tc::score_stats_tc<1>, mx) && set_smem(tc::score_stats_tc<2>, mx) &&
-                  set_smem(tc::score_emit_tc<1>, mx) && set_smem(tc::score_emit_tc<2>, mx);
+                  set_smem(tc::score_emit_tc<1>, mx) && set_smem(tc::score_emit_tc<2>, mx) &&
+                  set_smem(tc::score_fused_tc<1>, mx) && set_smem(tc::score_fused_tc<2>, mx);
         }))
         return GRAPHKV_ERR_CUDA;
     const int tiles_stats = ceil_div(d.L, tc::kTileKeys), tiles_emit = ceil_div(d.N, tc::kTileKeys);
@@ -479,6 +480,17 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
         ea.zero = ex.zero;
         ea.zero_words = ex.zero_words;
         ea.local_hist = ex.k > 0 ? 1 : 0;
+        // one kernel for both sweeps when all its CTAs are resident at once (one per SM): the CTAs
+        // of a unit wait for one another between the passes
+        if (ex.k == 0 && nu * chunks_s <= sm_count() && !env_int("GRAPHKV_TWO_SCORE_KERNELS", 0)) {
+            tc::ScoreTcArgs fa = ea;
+            fa.chunks = chunks_s;
+            fa.n_tiles = tiles_stats;
+            fa.wait_prior = next_launch_is_dependent();
+            rc = launch_ex("score_fused_tc", row_tiles == 1 ? tc::score_fused_tc<1> : tc::score_fused_tc<2>,
+                           dim3(chunks_s, nu), dim3(tc::kScoreThreads), smem, st, fa.wait_prior != 0, 1, tmK, fa);
+            continue;
+        }
         sa.wait_prior = next_launch_is_dependent();
         rc = launch_ex("score_stats_tc", row_tiles == 1 ? tc::score_stats_tc<1> : tc::score_stats_tc<2>,
                        dim3(chunks_s, nu), dim3(tc::kScoreThreads), smem, st, sa.wait_prior != 0, 1, tmK, sa);

@@ -37,7 +37,9 @@ struct ScoreTcArgs {
     const __nv_bfloat16 *Q;
     float *part;        // [units][stats_chunks][GW][2] row statistics (max, sum) per key chunk
     float *row_c;       // [units][GW] c_r = max_r + log2(Z_r), written by the last stats CTA of a unit
-    int *arrivals;      // [units] stats CTAs done per unit (zero before the launch; reset on the way)
+    int *arrivals;      // [2 * units] counters of CTAs per unit (zero before the launch; reset on the way):
+                        // the two-kernel path counts finished statistics CTAs in [unit], the kernel of
+                        // both sweeps arrivals and departures of its hand-over in [2 * unit], [2 * unit + 1]
     float *a_out;       // [units][N] attention mass before pooling
     uint32_t *a_hist;   // optional [units][kMassBins]: counts of a by the top bits of its ordered image
     int *status;        // workspace status word
@@ -54,8 +56,9 @@ struct ScoreTcArgs {
     int zero_words;
     int local_hist;     // build the per-CTA mass histogram even without a_hist
     long long wait_cycles;   // limit of every wait of the kernel, in clocks
-    int withhold_commit;     // test hook (statistics sweep): the MMA issuer leaves out the arrival that
-                             // announces its first accumulator, so the wait for it runs out
+    int withhold_commit;     // test hook (statistics sweep): 1: the MMA issuer leaves out the arrival that
+                             // announces its first accumulator, so the wait for it runs out; 2 (kernel of
+                             // both sweeps): no CTA announces itself at the hand-over, so that wait runs out
 };
 
 struct ScoreSmem {
@@ -185,6 +188,39 @@ __device__ __forceinline__ void stats_fold(float (&v)[32], float scale, float &m
     z += ex2_sum32(v, pack2(scale, scale), [&](int) { return make_ulonglong2(nm, nm); });
 }
 
+// (max, sum) of a row over the partials of all key chunks of a unit: kTpr consecutive threads of a
+// warp share the row, thread `sub` of them takes chunks sub, sub + kTpr, ..., eight loads in flight,
+// and the shares are combined with shuffles (every thread of the warp calls this).  Both score
+// paths merge this way, so they agree to the bit.
+template <int kTpr>
+__device__ __forceinline__ float2 merge_row_partials(const float2 *pu, int chunks, int GW, int r, int sub)
+{
+    float mx = kNegBig, z = 0.f;
+    if (r < GW) {
+        for (int q0 = sub; q0 < chunks; q0 += 8 * kTpr) {
+            float2 v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                v[k] = q0 + k * kTpr < chunks ? __ldcg(pu + (long long)(q0 + k * kTpr) * GW + r)
+                                              : make_float2(kNegBig, 0.f);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float mn = fmaxf(mx, v[k].x);
+                z = z * ex2(mx - mn) + v[k].y * ex2(v[k].x - mn);
+                mx = mn;
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 1; o < kTpr; o <<= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, mx, o), z2 = __shfl_xor_sync(0xffffffffu, z, o);
+        const float mn = fmaxf(mx, m2);
+        z = z * ex2(mx - mn) + z2 * ex2(m2 - mn);
+        mx = mn;
+    }
+    return make_float2(mx, z);
+}
+
 // kRowTiles = 1 (G*W <= 128) or 2 (G*W <= 256).  grid (chunks, units of the launch).
 template <int kRowTiles>
 __global__ void __launch_bounds__(kScoreThreads, 1)
@@ -254,7 +290,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
                     }
                 }
                 umma_commit(s.empty0 + 8 * st);
-                if (!(a.withhold_commit && i == 0)) umma_commit(s.tfull0 + 8 * buf);
+                if (!(a.withhold_commit == 1 && i == 0)) umma_commit(s.tfull0 + 8 * buf);
             }
         }
     } else {
@@ -338,22 +374,11 @@ score_stats_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     if (*s_flag) {
         __threadfence();
         const float2 *pu = reinterpret_cast<const float2 *>(a.part) + (long long)unit * a.stats_chunks * d.GW;
-        for (int r = threadIdx.x; r < d.GW; r += kScoreThreads) {
-            float mx = kNegBig, z = 0.f;
-            for (int q0 = 0; q0 < a.chunks; q0 += 8) {       // eight loads in flight at a time
-                float2 v[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    v[k] = q0 + k < a.chunks ? __ldcg(pu + (long long)(q0 + k) * d.GW + r)
-                                             : make_float2(kNegBig, 0.f);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float mn = fmaxf(mx, v[k].x);
-                    z = z * ex2(mx - mn) + v[k].y * ex2(v[k].x - mn);
-                    mx = mn;
-                }
-            }
-            a.row_c[(long long)unit * d.GW + r] = mx + log2f(z);
+        constexpr int kTpr = 4 / kRowTiles;
+        if (threadIdx.x < kRowsPad * kTpr) {
+            const int r = threadIdx.x / kTpr, sub = threadIdx.x % kTpr;
+            const float2 mz = merge_row_partials<kTpr>(pu, a.chunks, d.GW, r, sub);
+            if (sub == 0 && r < d.GW) a.row_c[(long long)unit * d.GW + r] = mz.x + log2f(mz.y);
         }
         if (threadIdx.x == 0) a.arrivals[unit] = 0;      // ready for the next launch
     }
@@ -536,6 +561,337 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
                           a.a_out + (long long)unit * d.N, mass_hist, gen + (s.stage0 - s.q));
     pc.mark();
     pc.flush(1);
+}
+
+
+// Both sweeps in one kernel, for launches whose CTAs are all resident at once (one CTA per SM and
+// no more CTAs than SMs): a CTA runs the statistics pass over its key chunk, leaves its partial
+// row statistics, announces itself on the unit's counter, waits (bounded, like every wait here)
+// until all chunks of the unit have done so, merges the partials into the row constants itself
+// and runs the emit pass over the same chunk in reverse tile order, so that the tiles the first
+// pass left in the stage ring are used again without a copy.  Against two launches this saves a
+// kernel boundary, the second set-up (barriers, tensor memory, the staging of the queries) and
+// the re-read of the ring's tiles.  kTiles = 1 (G*W <= 128) or 2 (G*W <= 256); grid (chunks,
+// units of the launch); a.arrivals holds two counters per unit (arrived, departed), zero before
+// the launch and zero again after it.
+template <int kTiles>
+__global__ void __launch_bounds__(kScoreThreads, 1)
+score_fused_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    PhaseClock pc(threadIdx.x == 64);
+    pc.mark();
+    constexpr int kRowsPad = 128 * kTiles;
+    constexpr int kBufCols = 128 * kTiles;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr int kBufs = 512 / kBufCols, kGroups = 2 / kTiles, kSets = 4 / kGroups;
+    constexpr int kXchg = 16 / kSets;
+    constexpr int kParts = 4 / kTiles;               // partial statistics per row within the CTA
+    const Dims &d = a.d;
+    const long long lim = a.wait_cycles;
+    uint8_t *gen;
+    const ScoreSmem s = score_smem_layout(smem_raw, kRowsPad, a.stages, &gen);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int unit = a.unit0 + blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
+    const int chunk = blockIdx.x;
+    const int S = a.stages;
+    int t0, t1;
+    tile_range(a.n_tiles, a.chunks, chunk, &t0, &t1);
+    const int n_local = t1 - t0;                                          // tiles of the statistics pass
+    const int n_emit = max(0, min(t1, ceil_div(d.N, kTileKeys)) - t0);    // of them, tiles with prefix keys
+    const int n_cols = (d.GW + 31) & ~31;            // UMMA N of the emit pass
+
+    // scratch: first the CTA's partial statistics, after the hand-over the row constants and the
+    // exchange buffers of the emit pass
+    float2 *cta_part = reinterpret_cast<float2 *>(gen + (s.misc - s.q));      // [kParts][kRowsPad]
+    float *row_c = reinterpret_cast<float *>(gen + (s.misc - s.q));           // [kRowsPad]
+    float *xchg = row_c + 256;                                                // [kXchg tiles][kSets][128]
+    uint32_t *mass_hist = reinterpret_cast<uint32_t *>(gen + (s.misc - s.q) + kScratchBytes);   // [kMassBins]
+    int *s_flag = reinterpret_cast<int *>(gen + (s.tmem_slot - s.q)) + 2;
+    const int n_ahead = min(n_local, S);
+
+    const uint32_t tmem_base = score_setup(s, gen, &tmK, S, kTmemCols, kEpiWarps / kGroups);
+    bool ok = true;
+    if (warp == 0) {
+        if (lane == 0) ok = score_produce(s, &tmK, S, t0, 0, n_ahead, h, b, lim);
+    } else {
+        stage_q(gen, kRowsPad, d, a.Q, b, h, threadIdx.x - 32, kScoreThreads - 32);
+        fence_proxy_async();
+    }
+    pc.mark();
+    if (a.wait_prior) pdl_wait();
+    pc.mark();
+    pdl_launch_dependents();
+    const bool want_hist = a.a_hist != nullptr || a.local_hist;
+    if (want_hist)
+        for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads) mass_hist[i] = 0u;
+    if (a.zero) {
+        const int per_cta = ceil_div(a.zero_words, a.chunks);
+        for (int i = chunk * per_cta + threadIdx.x; i < min((chunk + 1) * per_cta, a.zero_words); i += kScoreThreads)
+            a.zero[(long long)unit * a.zero_words + i] = 0u;
+    }
+    __syncthreads();
+    pc.mark();
+
+    // ---- statistics pass: D = Q K^T, tiles 0 .. n_local-1 in order ----
+    if (warp == 0) {
+        if (lane == 0 && ok) ok = score_produce(s, &tmK, S, t0, n_ahead, n_local, h, b, lim);
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
+            for (int i = 0; i < n_local; ++i) {
+                const int st = i % S, ph = (i / S) & 1;
+                const int buf = i % kBufs, bph = (i / kBufs) & 1;
+                if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1, lim)) { ok = false; break; }
+                if (!mbar_wait(s.full0 + 8 * st, ph, lim)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t kt = s.stage0 + st * kTileBytes;
+#pragma unroll
+                for (int rt = 0; rt < kTiles; ++rt) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t koff = (k >> 2) * kHalfBytes + (k & 3) * 32;
+                        const uint32_t qoff = (k >> 2) * (kRowsPad * 128) + rt * (128 * 128) + (k & 3) * 32;
+                        umma_bf16(tmem_base + buf * kBufCols + rt * 128, umma_desc_sw128(s.q + qoff),
+                                  umma_desc_sw128(kt + koff), idesc, k > 0);
+                    }
+                }
+                umma_commit(s.empty0 + 8 * st);
+                if (!(a.withhold_commit == 1 && i == 0)) umma_commit(s.tfull0 + 8 * buf);
+            }
+        }
+    } else {
+        constexpr int kSetCols = 64;
+        const int quad = warp & 3, set = (warp - 2) >> 2;
+        const int grp = set / (4 / kGroups);
+        const int row = quad * 32 + lane;
+        const int col0 = (set % (4 / kGroups)) * kSetCols, rt = col0 >> 7, key_off = col0 & 127;
+        const float scale = rsqrtf((float)kHeadDim) * kLog2e;
+        float mx = kNegBig, z = 0.f;
+        const int r = rt * 128 + row;
+        const int last = d.N + (r < d.GW ? r % d.W : 0);      // last visible key of the row
+        bool alive = true;
+        for (int i = grp; i < n_local && alive; i += kGroups) {
+            const int buf = i % kBufs, bph = (i / kBufs) & 1;
+            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, bph, lim));
+            if (!alive) break;
+            tc_fence_after();
+            uint32_t raw[kSetCols / 32][32];
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kBufCols + col0;
+#pragma unroll
+            for (int c = 0; c < kSetCols / 32; ++c) tmem_ld32_issue(t_row + c * 32, raw[c]);
+#pragma unroll
+            for (int c = 0; c < kSetCols / 32; ++c) tmem_ld_fence(raw[c]);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s.tempty0 + 8 * buf);
+            const int key0 = (t0 + i) * kTileKeys + key_off;
+            const bool masked = key0 + kSetCols - 1 > d.N;      // window keys or the tail past L
+#pragma unroll
+            for (int c = 0; c < kSetCols / 32; ++c) {
+                float v[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(raw[c][e]);
+                if (masked) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (key0 + c * 32 + e > last) v[e] = -INFINITY;
+                }
+                stats_fold(v, scale, mx, z);
+            }
+        }
+        ok = alive;
+        cta_part[(kTiles == 1 ? set : set & 1) * kRowsPad + r] = make_float2(mx, z);
+    }
+    pc.mark();
+
+    // ---- hand-over: partials out, every chunk of the unit in, row constants ----
+    tc_fence_before();
+    bool all_ok = __syncthreads_and(ok ? 1 : 0) != 0;
+    for (int r = threadIdx.x; r < d.GW; r += kScoreThreads) {
+        float2 p[kParts];
+        float mx = kNegBig;
+#pragma unroll
+        for (int k = 0; k < kParts; ++k) {
+            p[k] = cta_part[k * kRowsPad + r];
+            mx = fmaxf(mx, p[k].x);
+        }
+        float z = 0.f;
+#pragma unroll
+        for (int k = 0; k < kParts; ++k) z += p[k].y * ex2(p[k].x - mx);
+        reinterpret_cast<float2 *>(a.part)[((long long)unit * a.stats_chunks + chunk) * d.GW + r] =
+            make_float2(mx, z);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        // a CTA whose pass failed still arrives, so that the others do not wait for it in vain
+        int *arrived = a.arrivals + 2 * unit;
+        if (a.withhold_commit != 2) atomicAdd(arrived, 1);
+        bool in = false;
+        const long long c0 = clock64();
+        while (true) {
+            int seen;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(arrived) : "memory");
+            if (seen >= a.chunks) { in = true; break; }
+            if (clock64() - c0 > lim) break;
+            __nanosleep(20);
+        }
+        *s_flag = in ? 1 : 0;
+    }
+    __syncthreads();
+    pc.mark();
+    if (!*s_flag) { ok = false; all_ok = false; }
+    if (all_ok) {
+        // every CTA merges the unit's partials itself: kTpr threads per row take the chunks in turn
+        constexpr int kTpr = 4 / kTiles;
+        const float2 *pu = reinterpret_cast<const float2 *>(a.part) + (long long)unit * a.stats_chunks * d.GW;
+        static_assert(kRowsPad * kTpr <= (kScoreThreads & ~31), "whole warps take the rows");
+        if (threadIdx.x < kRowsPad * kTpr) {
+            const int r = threadIdx.x / kTpr, sub = threadIdx.x % kTpr;
+            const float2 mz = merge_row_partials<kTpr>(pu, a.chunks, d.GW, r, sub);
+            // -c_r of the unit's rows; padding rows contribute 2^-inf = 0
+            if (sub == 0) row_c[r] = r < d.GW ? -(mz.x + log2f(mz.y)) : -INFINITY;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        // the last CTA of the unit to leave the hand-over clears both counters for the next launch
+        int *cnt = a.arrivals + 2 * unit;
+        if (atomicAdd(cnt + 1, 1) == a.chunks - 1) {
+            atomicExch(cnt, 0);
+            atomicExch(cnt + 1, 0);
+        }
+    }
+    pc.mark();
+
+    // ---- emit pass: D = K Q^T, the chunk's prefix tiles in reverse order ----
+    // Tile tl sits in ring slot tl % S in both passes; uses(st) counts the fills of slot st by the
+    // first pass, so the u-th use of a slot keeps the parities of its barriers in step.
+    auto slot_use = [&](int tl, int k) { return (n_local - (tl % S) + S - 1) / S + k / S; };
+    if (!all_ok) {
+        // nothing more to do: a wait ran out somewhere
+    } else if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int k = 0; k < n_emit; ++k) {
+                const int tl = n_emit - 1 - k, st = tl % S, u = slot_use(tl, k);
+                if (!mbar_wait(s.empty0 + 8 * st, (u & 1) ^ 1, lim)) { ok = false; break; }
+                if (tl + S >= n_local) {
+                    mbar_arrive(s.full0 + 8 * st);            // still there from the first pass
+                } else {
+                    const uint32_t dst = s.stage0 + st * kTileBytes;
+                    mbar_expect_tx(s.full0 + 8 * st, kTileBytes);
+                    tma_load_4d(dst, &tmK, s.full0 + 8 * st, 0, (t0 + tl) * kTileKeys, h, b);
+                    tma_load_4d(dst + kHalfBytes, &tmK, s.full0 + 8 * st, 64, (t0 + tl) * kTileKeys, h, b);
+                }
+                ++issued;
+            }
+            if (!ok)        // gave up: let the copies already in flight land before the CTA exits
+                for (int k = max(0, issued - S); k < issued; ++k) {
+                    const int tl = n_emit - 1 - k;
+                    mbar_wait(s.full0 + 8 * (tl % S), slot_use(tl, k) & 1, lim);
+                }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(128, n_cols);
+            for (int k = 0; k < n_emit; ++k) {
+                const int tl = n_emit - 1 - k, st = tl % S, u = slot_use(tl, k);
+                const int i = n_local + k;                        // accumulator buffers keep rotating
+                const int buf = i % kBufs, bph = (i / kBufs) & 1;
+                if (!mbar_wait(s.tempty0 + 8 * buf, bph ^ 1, lim)) { ok = false; break; }
+                if (!mbar_wait(s.full0 + 8 * st, u & 1, lim)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t kt = s.stage0 + st * kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t koff = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                    const uint32_t qoff = (kk >> 2) * (kRowsPad * 128) + (kk & 3) * 32;
+                    umma_bf16(tmem_base + buf * kBufCols, umma_desc_sw128(kt + koff),
+                              umma_desc_sw128(s.q + qoff), idesc, kk > 0);
+                }
+                umma_commit(s.empty0 + 8 * st);
+                umma_commit(s.tfull0 + 8 * buf);
+            }
+        }
+    } else {
+        const int quad = warp & 3, set = (warp - 2) >> 2;
+        const int grp = set / kSets, part = set % kSets;
+        const int key_lane = quad * 32 + lane;
+        const float scale = rsqrtf((float)kHeadDim) * kLog2e;
+        const uint64_t scale2 = pack2(scale, scale);
+        const int n_slices = (d.GW + 31) >> 5;
+        const int s_begin = (part * n_slices) / kSets, s_end = ((part + 1) * n_slices) / kSets;
+        float *a_row = a.a_out + (long long)unit * d.N;
+        const uint32_t t_set = tmem_base + ((uint32_t)(quad * 32) << 16) + s_begin * 32;
+        bool alive = true;
+        auto sum_slice = [&](const uint32_t (&reg)[32], int sl) {
+            float v[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(reg[e]);
+            const ulonglong2 *c4 = reinterpret_cast<const ulonglong2 *>(row_c + sl * 32);
+            return ex2_sum32(v, scale2, [&](int q) { return c4[q]; });
+        };
+        for (int k = grp; k < n_emit && alive; k += kGroups) {
+            const int i = n_local + k, buf = i % kBufs;
+            alive = __all_sync(0xffffffffu, mbar_wait(s.tfull0 + 8 * buf, (i / kBufs) & 1, lim));
+            if (!alive) break;
+            tc_fence_after();
+            auto release = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s.tempty0 + 8 * buf);
+            };
+            float acc = 0.f;
+            if (s_end - s_begin == 2) {
+                uint32_t ra[32], rb[32];
+                tmem_ld32_issue(t_set + buf * kBufCols, ra);
+                tmem_ld32_issue(t_set + buf * kBufCols + 32, rb);
+                tmem_ld_fence(ra);
+                tmem_ld_fence(rb);
+                release();
+                acc = sum_slice(ra, s_begin) + sum_slice(rb, s_begin + 1);
+            } else if (s_end - s_begin == 1) {
+                uint32_t ra[32];
+                tmem_ld32_issue(t_set + buf * kBufCols, ra);
+                tmem_ld_fence(ra);
+                release();
+                acc = sum_slice(ra, s_begin);
+            } else {
+                release();
+            }
+            // the sets of the tile exchange the parts of each key's row sum (see score_emit_tc)
+            const int xb = k % kXchg;
+            xchg[(xb * kSets + part) * 128 + key_lane] = acc;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s.xbar0 + 8 * xb);
+            if (part != (k / kGroups) % kSets) continue;
+            alive = __all_sync(0xffffffffu, mbar_wait(s.xbar0 + 8 * xb, (k / kXchg) & 1, lim));
+            const int j = (t0 + n_emit - 1 - k) * kTileKeys + key_lane;
+            if (alive && j < d.N) {
+                const float *x = xchg + xb * kSets * 128 + key_lane;
+                const float aj = kSets == 4 ? (x[0] + x[128]) + (x[256] + x[384]) : x[0] + x[128];
+                a_row[j] = aj;
+                if (want_hist) atomicAdd(&mass_hist[float_to_key(aj) >> 21], 1u);
+            }
+        }
+        ok = alive;
+    }
+    pc.mark();
+    if (!ok && a.status) atomicExch(a.status, (int)GRAPHKV_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (a.a_hist)
+        for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads)
+            if (mass_hist[i]) atomicAdd(a.a_hist + (long long)unit * kMassBins + i, mass_hist[i]);
+    pc.mark();
+    pc.flush(5);
 }
 
 }  // namespace tc

@@ -219,11 +219,13 @@ def test_identical_keys_take_the_exact_tie_paths(gk):
 
 @pytest.mark.parametrize("env", [{"GRAPHKV_NO_CLUSTER": "1"}, {"GRAPHKV_FORCE_SIMT": "1"},
                                  {"GRAPHKV_NO_CLUSTER": "1", "GRAPHKV_FORCE_SIMT": "1"},
-                                 {"GRAPHKV_L2_GROUP_MB": "1"}, {"GRAPHKV_TAIL_SOURCES": "1"},
+                                 {"GRAPHKV_L2_GROUP_MB": "1"}, {"GRAPHKV_TWO_SCORE_KERNELS": "1"},
+                                 {"GRAPHKV_TAIL_SOURCES": "1"},
                                  {"GRAPHKV_TAIL_SOURCES": "1", "GRAPHKV_NO_CLUSTER": "1"}])
 def test_fallback_kernels_agree_with_the_oracle(gk, env):
     # the generic row kernels (rows too long for a cluster), the SIMT sweeps (fp32 inputs, many
-    # sources or neighbours), several launch groups, and the source selection at the tail of the
+    # sources or neighbours), several launch groups, the two score sweeps as kernels of their own
+    # (launches with more CTAs than SMs), and the source selection at the tail of the
     # emit sweep with pooling in the finishing kernel, forced here on a case the fast path covers
     cfg = wl.scaled(wl.LLAMA_32K, n_prefix=4500, budget=300, n_q_heads=8, n_kv_heads=2,
                     n_clusters=32, neighbors=8, batch=2)
@@ -237,6 +239,30 @@ def test_fallback_kernels_agree_with_the_oracle(gk, env):
                 os.environ.pop(k, None)
             else:
                 os.environ[k] = v
+
+@pytest.mark.parametrize("window", [32, 64])
+def test_one_score_kernel_and_two_agree_to_the_bit(gk, window):
+    # the kernel that runs both sweeps (launches whose CTAs are all resident) and the two-kernel
+    # path merge the row statistics in the same order: identical scores
+    dev = torch.device("cuda:0")
+    cfg = wl.scaled(wl.LLAMA_32K, n_prefix=9000 + 37, budget=128, n_q_heads=8, n_kv_heads=2,
+                    n_clusters=32, window=window)
+    inp = wl.make_inputs(cfg)
+    Qd, Kd = inp["Qw"].to(dev), inp["K"].to(dev)
+    p = gk.make_params(Kd, Qw=Qd, window=cfg.window, pool_kernel=cfg.pool_kernel)
+    ws = gk.alloc_workspace(p, dev)
+    one = torch.empty((p.batch, p.n_kv_heads, cfg.n_prefix), dtype=torch.float32, device=dev)
+    two = torch.empty_like(one)
+    gk.graphkv_score(p, Qd, Kd, one, ws)
+    os.environ["GRAPHKV_TWO_SCORE_KERNELS"] = "1"
+    try:
+        gk.graphkv_score(p, Qd, Kd, two, ws)
+    finally:
+        os.environ.pop("GRAPHKV_TWO_SCORE_KERNELS", None)
+    assert gk.graphkv_read_status(ws) == gk.OK
+    assert torch.equal(one, two)
+    want = okv.score(inp["Qw"], inp["K"], cfg.window, cfg.pool_kernel)
+    assert pu.score_rel_err(one.cpu(), want) <= pu.SCORE_RTOL
 
 
 @pytest.mark.parametrize("case", [
