@@ -61,7 +61,7 @@ template <int NP> __host__ __device__ constexpr int sim_tiles_cap() { return 512
 template <int NP> __host__ __device__ inline size_t sim_smem_bytes(int stages)
 {
     return 1024 + (size_t)NP * 256 + (size_t)stages * kTileBytes + (8 + 8 + kSimMaxTiles) * 8 + 16 +
-           (size_t)sim_tiles_cap<NP>() * 128 * 4 + (size_t)NP * 5 * 4 + (size_t)NP * kCandCap * 8 + 64;
+           (size_t)sim_tiles_cap<NP>() * 128 * 4 + (size_t)NP * 6 * 4 + (size_t)NP * kCandCap * 8 + 64;
 }
 
 template <int NP>
@@ -98,13 +98,14 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
     const uint32_t s_tmem = s_done0 + kSimMaxTiles * 8;
     const uint32_t s_invn = s_tmem + 16;
     const uint32_t s_book = s_invn + kTilesCap * 128 * 4;
-    const uint32_t s_list = s_book + NP * 5 * 4;
+    const uint32_t s_list = s_book + NP * 6 * 4;
     float *inv_norm = reinterpret_cast<float *>(gen + (s_invn - base));        // [tile][128]
     int *src_pos = reinterpret_cast<int *>(gen + (s_book - base));              // [NP]
     float *src_inv = reinterpret_cast<float *>(src_pos + NP);                   // [NP]
     float *tau = src_inv + NP;                                                  // [NP] threshold cosine
     int *cnt = reinterpret_cast<int *>(tau + NP);                               // [NP]
     int *tau_bin = cnt + NP;                                                    // [NP] bin whose lower edge tau is
+    float *src_norm = reinterpret_cast<float *>(tau_bin + NP);                  // [NP] max(|k_c|, eps)
     Cand *list = reinterpret_cast<Cand *>(gen + (s_list - base));               // [NP][kCandCap]
     // after the sweep the stage memory holds the bins of the maxima and the threads' edge queues
     // (a key position takes 26 bits there: rows this kernel is given are shorter than 2^18 keys)
@@ -185,6 +186,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
         for (int o = 8; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
         if (in && c16 == 0) {
             src_pos[r] = pos;
+            src_norm[r] = fmaxf(sqrtf(n2), kNormEps);
             src_inv[r] = 1.0f / fmaxf(sqrtf(n2), kNormEps);
             cnt[r] = 0;
         }
@@ -289,7 +291,7 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             // 1. thresholds.  The cosine of a thread's best key for source c is the rounded product
             //    of its best dot / |k_j| with 1 / |k_c| (rounding is monotone).  Every thread leaves
             //    the cosine bins (of kMaxBins over [-1, 1]) of its maxima, four sources to a word; a
-            //    warp takes four sources and finds for each, by bisection over the bin index, the
+            //    warp takes two sources at a time and finds for each, by bisection over the bin index, the
             //    highest bin with m+1 maxima in or above it; tau is that bin's lower edge.
             //    (A thread without keys counts in bin 0, which only matters when tau is -1 anyway.)
 #pragma unroll
@@ -310,7 +312,8 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             asm volatile("bar.sync 1, 256;" ::: "memory");
             pc.mark();
             const int ew = warp - 2;
-            for (int g = ew; g * 4 < n_src; g += 8) {
+            for (int pr = ew; pr * 2 < n_src; pr += 8) {
+                const int g = pr >> 1, sh = (pr & 1) * 16;       // the pair's word and its two bytes there
                 uint32_t w8[8];              // this lane's eight threads' bins of sources 4g .. 4g+3
                 {
                     const uint4 lo = *reinterpret_cast<const uint4 *>(max_bin + g * kSimEpiThreads + lane * 8);
@@ -318,27 +321,26 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                     w8[0] = lo.x; w8[1] = lo.y; w8[2] = lo.z; w8[3] = lo.w;
                     w8[4] = hi.x; w8[5] = hi.y; w8[6] = hi.z; w8[7] = hi.w;
                 }
-                uint32_t bstar[4] = {0u, 0u, 0u, 0u};
+                uint32_t bstar[2] = {0u, 0u};
 #pragma unroll
                 for (int bit = 7; bit >= 0; --bit) {
-                    int n[4];
+                    int n[2];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
+                    for (int q = 0; q < 2; ++q) {
                         const uint32_t cand = bstar[q] | (1u << bit);
                         n[q] = 0;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) n[q] += ((w8[k] >> (8 * q)) & 0xffu) >= cand ? 1 : 0;
+                        for (int k = 0; k < 8; ++k) n[q] += ((w8[k] >> (sh + 8 * q)) & 0xffu) >= cand ? 1 : 0;
                     }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) n[q] = __reduce_add_sync(0xffffffffu, n[q]);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        if (n[q] >= d.m + 1) bstar[q] |= 1u << bit;
+                    // both counts in one reduction (each at most 256)
+                    const uint32_t both = __reduce_add_sync(0xffffffffu, (uint32_t)n[0] | ((uint32_t)n[1] << 16));
+                    if ((int)(both & 0xffffu) >= d.m + 1) bstar[0] |= 1u << bit;
+                    if ((int)(both >> 16) >= d.m + 1) bstar[1] |= 1u << bit;
                 }
-                if (lane < 4 && g * 4 + lane < n_src) {
-                    const uint32_t bs = lane == 0 ? bstar[0] : lane == 1 ? bstar[1] : lane == 2 ? bstar[2] : bstar[3];
-                    tau[g * 4 + lane] = bs == 0 ? -1.0f : (float)bs * (2.0f / kMaxBins) - 1.0f;
-                    tau_bin[g * 4 + lane] = (int)bs;
+                if (lane < 2 && pr * 2 + lane < n_src) {
+                    const uint32_t bs = lane == 0 ? bstar[0] : bstar[1];
+                    tau[pr * 2 + lane] = bs == 0 ? -1.0f : (float)bs * (2.0f / kMaxBins) - 1.0f;
+                    tau_bin[pr * 2 + lane] = (int)bs;
                 }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -354,20 +356,28 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             float theta[NP];
 #pragma unroll
             for (int c = 0; c < NP; ++c) {
-                const float q = c < n_src ? (tau[c] - 2.4e-7f) / src_inv[c] : INFINITY;
-                theta[c] = q - fabsf(q) * 2.4e-7f - 1e-30f;
+                // (times the norm instead of divided by its rounded reciprocal: within 1.2e-7 of it,
+                // inside the margin taken off below)
+                const float q = c < n_src ? (tau[c] - 2.4e-7f) * src_norm[c] : INFINITY;
+                theta[c] = q - fabsf(q) * 3.6e-7f - 1e-30f;
             }
-            // (branch-free, the store and the count under one predicate; a key past the end of the
-            // row gets a NaN factor, which fails every comparison)
+            // (the store and the count under one predicate; a key past the end of the row gets a NaN
+            // factor, which fails every comparison)
             uint2 *const q0 = queue + et;
             const uint32_t q_first = smem_u32(q0), q_step = kSimEpiThreads * sizeof(uint2);
             const uint32_t q_last = q_first + (kQueueCap - 1) * q_step;
             uint32_t qa = q_first;
-            for (int i = set; i < n_local; i += 2) {
+            auto list_tile = [&](int i, const float (&v)[NP]) {
                 const int j = (t0 + i) * kTileKeys + key_lane;
                 const float inv = j < d.N ? inv_norm[i * 128 + key_lane] : __int_as_float(0x7fc00000);
-                float v[NP];
-                tmem_ld_np<NP>(lane_addr + i * NP, v);
+                // few keys pass any threshold: the independent comparisons first, the appends (a
+                // dependent chain through the queue's address) only for a key with an edge to list
+                if constexpr (NP <= 32) {
+                    bool any = false;
+#pragma unroll
+                    for (int c = 0; c < NP; ++c) any |= v[c] * inv >= theta[c];
+                    if (!any) return;
+                }
 #pragma unroll
                 for (int c = 0; c < NP; ++c) {
                     asm volatile(
@@ -380,6 +390,36 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
                         : "f"(v[c] * inv), "r"(((uint32_t)c << 26) | (uint32_t)j), "f"(theta[c]), "r"(q_last),
                           "r"(q_step)
                         : "memory");
+                }
+            };
+            if constexpr (NP <= 32) {
+                // the loads of two tiles are in flight together (a deeper unrolled body costs more in
+                // instruction fetches than it hides: the body runs a few times per CTA)
+                constexpr int kDepth = 2;
+                for (int i0 = set; i0 < n_local; i0 += 2 * kDepth) {
+                    uint32_t raw[kDepth][NP];
+#pragma unroll
+                    for (int q = 0; q < kDepth; ++q)
+                        if (i0 + 2 * q < n_local) {                  // uniform over the warp
+                            if constexpr (NP == 16) tmem_ld16_issue(lane_addr + (i0 + 2 * q) * NP, raw[q]);
+                            else tmem_ld32_issue(lane_addr + (i0 + 2 * q) * NP, raw[q]);
+                        }
+#pragma unroll
+                    for (int q = 0; q < kDepth; ++q) tmem_ld_fence(raw[q]);
+#pragma unroll
+                    for (int q = 0; q < kDepth; ++q)
+                        if (i0 + 2 * q < n_local) {
+                            float v[NP];
+#pragma unroll
+                            for (int c = 0; c < NP; ++c) v[c] = __uint_as_float(raw[q][c]);
+                            list_tile(i0 + 2 * q, v);
+                        }
+                }
+            } else {
+                for (int i = set; i < n_local; i += 2) {
+                    float v[NP];
+                    tmem_ld_np<NP>(lane_addr + i * NP, v);
+                    list_tile(i, v);
                 }
             }
             pc.mark();
