@@ -21,7 +21,8 @@ from . import binding as gk  # noqa: E402
 from . import workloads as wl  # noqa: E402
 
 KERNELS = {0: "score_stats_tc", 1: "score_emit_tc", 2: "similarity_tc", 3: "pool_select_kernel",
-           4: "finish_kernel (first CTA of a cluster)", 6: "finish_kernel (other CTAs)"}
+           4: "finish_kernel (first CTA of a cluster)", 5: "score_fused_tc",
+           6: "finish_kernel (other CTAs)"}
 
 
 def main(name: str = "llama31_8b_32k", steps: int = 5) -> None:
