@@ -162,8 +162,10 @@ graphkv_status graphkv_propagate(const graphkv_params *params, const void *K, fl
  * e_ij = cosine(x_i, y_j) with x the source node's row of tensor `src_tensor` and y the rows of
  * tensor `all_tensor` (graphkv_tensor: K or V, with the strides the params give for it).  K/K is
  * Eq. 1 and what graphkv_propagate computes; V/V and K/V are the value-to-value and key-to-value
- * variants.  (Query-to-key and query-to-query edges would need the queries of every prefix token,
- * which a prefill-time cache does not hold.)  A tensor that is not used may be NULL. */
+ * variants.  The two arguments are operands only: a caller that still holds the query vectors of
+ * every token (one vector per KV head and token, laid out like V: e.g. the mean over the head's
+ * query group) passes them as `V` to get query-to-key or query-to-query edges.  A tensor that is
+ * not used may be NULL. */
 graphkv_status graphkv_propagate_edges(const graphkv_params *params, const void *K, const void *V,
                                        int32_t src_tensor, int32_t all_tensor, float *scores,
                                        int32_t *src_idx_out, void *workspace,

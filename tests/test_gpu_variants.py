@@ -128,13 +128,18 @@ def test_average_pooling(gk, env_simt, monkeypatch):
     assert torch.equal(s2.cpu().view(torch.int32), s.cpu().view(torch.int32))
 
 
-@pytest.mark.parametrize("kinds", [("V", "V"), ("K", "V")])
+@pytest.mark.parametrize("kinds", [("V", "V"), ("K", "V"), ("Q", "K"), ("K", "Q")])
 @pytest.mark.parametrize("env_simt", [False, True])
 def test_value_edges(gk, kinds, env_simt, monkeypatch):
     if env_simt:
         monkeypatch.setenv("GRAPHKV_FORCE_SIMT", "1")
     cfg = small_cfg()
     inp = wl.make_inputs(cfg)
+    if "Q" in kinds:
+        # query-to-key edges: the caller hands the per-KV-head query vectors of every token in the
+        # argument named V (a second draw of the key recipe stands in for them here)
+        inp["V"] = wl.make_inputs(cfg, layer=1)["K"]
+        kinds = tuple("V" if k == "Q" else k for k in kinds)
     Qd, Kd, Vd = (inp[k].to(DEV) for k in ("Qw", "K", "V"))
     kw = kwargs(cfg)
     p = gk.make_params(Kd, Qw=Qd, V=Vd, **kw)
