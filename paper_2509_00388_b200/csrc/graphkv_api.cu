@@ -165,10 +165,12 @@ ClusterPlan cluster_plan(const Dims &d)
 {
     ClusterPlan p{false, 1, 0, (d.kp - 1) / 2};
     if (env_int("GRAPHKV_NO_CLUSTER", 0)) return p;
-    // as many CTAs per row as keep a chunk near 4096 scores, but all clusters in one wave of the
+    // as many CTAs per row as keep a chunk near 2048 scores (the gather of the kept rows is spread
+    // over the cluster's CTAs: 16384-score rows with 2048 kept rows finish in 35 us on 8 CTAs per
+    // row against 42 us on 4), but all clusters in one wave of the
     // 148 SMs when the rows allow it (two waves of clusters of 8 measured 1.8x slower than one
     // wave of clusters of 4 for 32 rows of 131072)
-    while (p.C < cs::kMaxCluster && ceil_div(d.N, p.C) > 4096) p.C *= 2;
+    while (p.C < cs::kMaxCluster && ceil_div(d.N, p.C) > 2048) p.C *= 2;
     while (p.C > 1 && d.units * p.C > sm_count() && ceil_div(d.N, p.C / 2) <= cs::kMaxChunk) p.C /= 2;
     // hundreds of sources: their neighbour lists are merged by groups of warps, kMergeWarps per CTA,
     // so more CTAs per row shorten that phase as long as all clusters stay in one wave
