@@ -63,7 +63,7 @@ class Report:
                 "notes": self.notes[:32]}
 
     def write(self, name: str) -> None:
-        """Leaves the counters on file (gpurun_out/parity_<name>.json under the repository)."""
+        """Leaves the counters on file: parity_<name>.json in the repository's scratch output folder."""
         out = os.path.join(ROOT, "gpurun_out")
         try:
             os.makedirs(out, exist_ok=True)
