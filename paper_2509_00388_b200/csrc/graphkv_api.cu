@@ -315,6 +315,11 @@ inline bool next_launch_is_dependent()
     return dep;
 }
 
+// Set before a launch_ex whose kernel makes its CTAs wait for one another: the launch then asks
+// for all CTAs of the grid to be resident together (a cooperative launch), so that no other work
+// on the device can keep part of the grid waiting for SMs that the rest of it holds.
+thread_local bool t_cooperative = false;
+
 template <typename... KArgs, typename... Args>
 graphkv_status launch_ex(const char *name, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
                          cudaStream_t st, bool dependent, int cluster_x, Args &&...args)
@@ -324,8 +329,14 @@ graphkv_status launch_ex(const char *name, void (*kern)(KArgs...), dim3 grid, di
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[3];
     int n = 0;
+    if (t_cooperative) {
+        t_cooperative = false;
+        attr[n].id = cudaLaunchAttributeCooperative;
+        attr[n].val.cooperative = 1;
+        ++n;
+    }
     if (cluster_x > 1) {
         attr[n].id = cudaLaunchAttributeClusterDimension;
         attr[n].val.clusterDim.x = cluster_x;
@@ -483,15 +494,20 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
         ea.zero_words = ex.zero_words;
         ea.local_hist = ex.k > 0 ? 1 : 0;
         // one kernel for both sweeps when all its CTAs are resident at once (one per SM): the CTAs
-        // of a unit wait for one another between the passes
+        // of a unit wait for one another between the passes, so the launch is a cooperative one
+        // (the device starts the grid only when all of it fits beside whatever else is running);
+        // a device that refuses it gets the two kernels
         if (ex.k == 0 && nu * chunks_s <= sm_count() && !env_int("GRAPHKV_TWO_SCORE_KERNELS", 0)) {
             tc::ScoreTcArgs fa = ea;
             fa.chunks = chunks_s;
             fa.n_tiles = tiles_stats;
             fa.wait_prior = next_launch_is_dependent();
+            t_cooperative = true;
             rc = launch_ex("score_fused_tc", row_tiles == 1 ? tc::score_fused_tc<1> : tc::score_fused_tc<2>,
                            dim3(chunks_s, nu), dim3(tc::kScoreThreads), smem, st, fa.wait_prior != 0, 1, tmK, fa);
-            continue;
+            if (rc == GRAPHKV_OK) continue;
+            cudaGetLastError();
+            rc = GRAPHKV_OK;
         }
         sa.wait_prior = next_launch_is_dependent();
         rc = launch_ex("score_stats_tc", row_tiles == 1 ? tc::score_stats_tc<1> : tc::score_stats_tc<2>,

@@ -565,7 +565,7 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
 
 
 // Both sweeps in one kernel, for launches whose CTAs are all resident at once (one CTA per SM and
-// no more CTAs than SMs): a CTA runs the statistics pass over its key chunk, leaves its partial
+// no more CTAs than SMs; launched cooperatively, so the device starts the grid as a whole): a CTA runs the statistics pass over its key chunk, leaves its partial
 // row statistics, announces itself on the unit's counter, waits (bounded, like every wait here)
 // until all chunks of the unit have done so, merges the partials into the row constants itself
 // and runs the emit pass over the same chunk in reverse tile order, so that the tiles the first
