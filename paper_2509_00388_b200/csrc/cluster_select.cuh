@@ -482,10 +482,12 @@ __device__ __forceinline__ Threshold cluster_kth_fine(cg::cluster_group &cl, int
 
 // Ascending positions of the kept elements of the cluster's row -> out[0..k).  Returns nothing;
 // ends with the writes of this CTA issued (callers fence before another CTA reads them).
-// One cluster barrier.
+// One cluster barrier.  `mirror` (optional): every kept position also goes into that array in the
+// shared memory of each of the cluster's `n_mirror` CTAs, complete after the cluster's next barrier.
 template <bool kListed>
 __device__ void cluster_emit_sorted_t(cg::cluster_group &cl, int C, int rank, const Smem &s,
-                                      const RowView &row, int base, Threshold th, int *out)
+                                      const RowView &row, int base, Threshold th, int *out,
+                                      int *mirror = nullptr, int n_mirror = 1)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_local = row.n;
@@ -545,17 +547,26 @@ __device__ void cluster_emit_sorted_t(cg::cluster_group &cl, int C, int rank, co
         const uint32_t gi = gt_before + __popc(bg & below), e = eq_before + __popc(be & below);
         const bool keep = is_gt || (is_eq && e < th.remaining);
         const int t = (int)(gi + min(e, th.remaining));
-        if (keep) out[t] = base + at;
+        if (keep) {
+            out[t] = base + at;
+            if (mirror) {
+                if (n_mirror > 1)
+                    for (int p = 0; p < n_mirror; ++p) cl.map_shared_rank(mirror, p)[t] = base + at;
+                else
+                    mirror[t] = base + at;
+            }
+        }
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
 }
 
 __device__ __forceinline__ void cluster_emit_sorted(cg::cluster_group &cl, int C, int rank, const Smem &s,
-                                                    const RowView &row, int base, Threshold th, int *out)
+                                                    const RowView &row, int base, Threshold th, int *out,
+                                                    int *mirror = nullptr, int n_mirror = 1)
 {
-    if (row.list) cluster_emit_sorted_t<true>(cl, C, rank, s, row, base, th, out);
-    else cluster_emit_sorted_t<false>(cl, C, rank, s, row, base, th, out);
+    if (row.list) cluster_emit_sorted_t<true>(cl, C, rank, s, row, base, th, out, mirror, n_mirror);
+    else cluster_emit_sorted_t<false>(cl, C, rank, s, row, base, th, out, mirror, n_mirror);
 }
 
 // The m largest edges (cosine descending, position ascending) of the lists when too many tie at
@@ -1291,6 +1302,11 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
 
     if (a.do_select) {
         int *idx = a.idx_out + (long long)unit * d.B;
+        // the kept positions also go into every CTA's shared memory (the fine histogram's words,
+        // idle by then), so that the gather neither waits for global writes of other CTAs to become
+        // visible nor for a load of the index ahead of every row
+        int *idx_s = reinterpret_cast<int *>(s.fine);
+        const bool mirrored = gathers && B <= kFineBins;
         if (holds) {
             // rank only the elements that reach a lower bound of the B-th largest, where one is at hand
             // (the staging arrays of the lists are free by now)
@@ -1306,14 +1322,16 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
             // (its threshold bin would hold too many elements to rank by counting)
             const Threshold th = sparse ? cluster_kth_fine(cl, R, rank, s, row, base, (uint32_t)B, pc)
                                         : cluster_kth(cl, R, rank, s, row, (uint32_t)B);
-            cluster_emit_sorted(cl, R, rank, s, row, base, th, idx);
+            cluster_emit_sorted(cl, R, rank, s, row, base, th, idx, mirrored ? idx_s : nullptr, C);
         }
         pc.mark();
-        __threadfence();
+        if (!mirrored) __threadfence();
         if (C > 1) cl.sync(); else __syncthreads();
         pc.mark();
         // gather: the cluster's threads share the 16-byte pieces of the B kept rows
-        if (gathers) copy_rows(0, (long long)B * 2 * vpr, [&](int t) { return (long long)__ldcg(idx + t); });
+        if (gathers)
+            copy_rows(0, (long long)B * 2 * vpr,
+                      [&](int t) { return (long long)(mirrored ? idx_s[t] : __ldcg(idx + t)); });
     }
     pc.mark();
     if (C > 1) cl.sync();      // no CTA leaves while its shared memory may still be read
