@@ -46,7 +46,7 @@ extern "C" {
 typedef enum {
     GRAPHKV_OK = 0,
     GRAPHKV_ERR_INVALID_ARG = 1,   /* NULL pointer, size or stride out of range, misalignment   */
-    GRAPHKV_ERR_UNSUPPORTED = 2,   /* valid but not implemented (head_dim != 128, G*W > 256, ...) */
+    GRAPHKV_ERR_UNSUPPORTED = 2,   /* valid but not implemented (head_dim not 128 or 64, G*W > 256, ...) */
     GRAPHKV_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small                 */
     GRAPHKV_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                          */
     GRAPHKV_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out (read_status only)      */
@@ -67,7 +67,7 @@ typedef struct {
     int32_t batch;        /* independent sequences (or any independent units sharing the shape)  */
     int32_t n_q_heads;
     int32_t n_kv_heads;   /* must divide n_q_heads                                               */
-    int32_t head_dim;     /* D; 128 required                                                     */
+    int32_t head_dim;     /* D: 128, or 64 (served by the general kernels, not the tensor cores) */
     int32_t seq_len;      /* L = N + W rows present in K and V                                   */
     int32_t window;       /* W >= 1 observation-window rows: queried from, always kept           */
     int32_t budget;       /* B = k_l: prefix tokens kept, 1 <= B <= N; outputs hold B + W rows   */

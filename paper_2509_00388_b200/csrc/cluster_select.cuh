@@ -1204,7 +1204,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
     pdl_launch_dependents();
     pc.mark();
     const int b = unit / d.hkv, h = unit % d.hkv;
-    const long long row_bytes = (long long)kHeadDim * a.elem_bytes;
+    const long long row_bytes = (long long)d.D * a.elem_bytes;
     const int rows_out = d.B + d.W;                        // rows the outputs hold per unit
     const int B = a.per_batch_budget ? a.budget_of[b] : d.B;   // this unit's budget
     const int vpr = (int)(row_bytes >> 4);                 // 16-byte pieces per row

@@ -9,7 +9,7 @@
 
 namespace graphkv {
 
-constexpr int kHeadDim = 128;          // D, fixed by the library
+constexpr int kHeadDim = 128;          // D of the tensor-core kernels (the SIMT kernels also take 64)
 constexpr int kMaxRows = 256;          // G*W limit (one TMEM accumulator tile of query rows)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegBig = -1.0e30f;    // finite stand-in for -inf in running maxima
@@ -18,6 +18,7 @@ constexpr float kNormEps = 1e-12f;     // floor of a key norm in Eq. 1
 // Shape of one call, resolved once on the host and passed by value to kernels.
 struct Dims {
     int batch, hq, hkv, G, W, N, L, GW;
+    int D;                     // head dimension: 128, or 64 (SIMT kernels only)
     int B, kp, K_src, m, T;
     float lambda;
     int units;                 // batch * hkv independent (sequence, KV head) problems

@@ -14,10 +14,10 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(
     Dims d, int elem_bytes, const unsigned char *__restrict__ K, const unsigned char *__restrict__ V,
     const int *__restrict__ idx, unsigned char *__restrict__ K_out, unsigned char *__restrict__ V_out)
 {
-    const int vec_per_row = kHeadDim * elem_bytes / 16;
+    const int vec_per_row = d.D * elem_bytes / 16;
     const long long rows_out = d.B + d.W;
     const long long total = (long long)d.units * rows_out * vec_per_row;
-    const long long row_bytes = (long long)kHeadDim * elem_bytes;
+    const long long row_bytes = (long long)d.D * elem_bytes;
     for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < total;
          p += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(p % vec_per_row);

@@ -64,7 +64,7 @@ graphkv_status resolve(const graphkv_params *p, Dims *d)
     if (p->pool_mode != GRAPHKV_POOL_MAX && p->pool_mode != GRAPHKV_POOL_AVG) return GRAPHKV_ERR_INVALID_ARG;
     if (p->signal < GRAPHKV_SIGNAL_DECAY || p->signal > GRAPHKV_SIGNAL_EVICT) return GRAPHKV_ERR_INVALID_ARG;
     if (p->reselect != 0 && p->reselect != 1) return GRAPHKV_ERR_INVALID_ARG;
-    if (p->head_dim != kHeadDim) return GRAPHKV_ERR_UNSUPPORTED;
+    if (p->head_dim != kHeadDim && p->head_dim != 64) return GRAPHKV_ERR_UNSUPPORTED;
     const int G = p->n_q_heads / p->n_kv_heads;
     if ((long long)G * p->window > kMaxRows) return GRAPHKV_ERR_UNSUPPORTED;
     if ((long long)p->batch * p->n_kv_heads > 65535) return GRAPHKV_ERR_UNSUPPORTED;
@@ -75,9 +75,9 @@ graphkv_status resolve(const graphkv_params *p, Dims *d)
         if (p->q_stride[i] % vec || p->k_stride[i] % vec || p->v_stride[i] % vec)
             return GRAPHKV_ERR_INVALID_ARG;
     }
-    if (p->q_stride[2] < kHeadDim || p->k_stride[2] < kHeadDim || p->v_stride[2] < kHeadDim)
+    if (p->q_stride[2] < p->head_dim || p->k_stride[2] < p->head_dim || p->v_stride[2] < p->head_dim)
         return GRAPHKV_ERR_INVALID_ARG;
-    d->batch = p->batch; d->hq = p->n_q_heads; d->hkv = p->n_kv_heads; d->G = G;
+    d->batch = p->batch; d->hq = p->n_q_heads; d->hkv = p->n_kv_heads; d->G = G; d->D = p->head_dim;
     d->W = p->window; d->L = p->seq_len; d->N = N; d->GW = G * p->window;
     d->B = p->budget; d->kp = p->pool_kernel; d->K_src = p->topk_nodes;
     d->m = graphkv_resolve_neighbors(N, p->neighbors);
@@ -128,7 +128,7 @@ int sm_count()
 // (GRAPHKV_L2_GROUP_MB bounds the keys of a group for experiments).
 int units_per_group(const Dims &d)
 {
-    const double mb = (double)d.L * kHeadDim * 2 / 1.0e6;
+    const double mb = (double)d.L * d.D * 2 / 1.0e6;
     int n = (int)(env_int("GRAPHKV_L2_GROUP_MB", 1 << 20) / mb);
     if (n < 1) n = 1;
     if (n > d.units) n = d.units;
@@ -196,7 +196,9 @@ struct SimPlan {
 SimPlan sim_plan(const Dims &d, bool bf16)
 {
     SimPlan p{false, 16, 1, ceil_div(d.N, tc::kTileKeys), 5};
-    if (!bf16 || d.K_src < 1 || d.K_src > kSimMaxSources || d.m < 1 || d.m > tc::kSimMaxNeighbors) return p;
+    if (!bf16 || d.D != kHeadDim || d.K_src < 1 || d.K_src > kSimMaxSources || d.m < 1 ||
+        d.m > tc::kSimMaxNeighbors)
+        return p;
     if (env_int("GRAPHKV_FORCE_SIMT", 0)) return p;
     if (!cluster_plan(d).ok) return p;          // its candidate lists are merged by the cluster kernel
     p.NP = d.K_src <= 16 ? 16 : (d.K_src <= 32 ? 32 : 64);
@@ -383,19 +385,28 @@ graphkv_status run_mass_simt(const Dims &d, const Layout &l, const T *Q, const T
 {
     float *part = at<float>(ws, l.part);
     const int threads = ceil_div(d.GW, 32) * 32;
-    GKV_LAUNCH("score_stats_simt", st,
-               (score_stats_simt<T><<<dim3(l.n_stat_chunks, d.units), threads, 0, st>>>(
-                   d, Q, K, part, l.n_stat_chunks, at<int>(ws, l.status))));
-    const size_t smem = ((size_t)d.GW * kHeadDim + 2 * d.GW) * sizeof(float);
+    const size_t smem = ((size_t)d.GW * d.D + 2 * d.GW) * sizeof(float);
     static std::mutex mu;
     static signed char state[64] = {};
     if (!once_per_device(mu, state, [] {
-            return set_smem(score_emit_simt<T>, ((size_t)kMaxRows * kHeadDim + 2 * kMaxRows) * sizeof(float));
+            const size_t mx = ((size_t)kMaxRows * kHeadDim + 2 * kMaxRows) * sizeof(float);
+            return set_smem(score_emit_simt<T, 128>, mx) && set_smem(score_emit_simt<T, 64>, mx);
         }))
         return GRAPHKV_ERR_CUDA;
-    GKV_LAUNCH("score_emit_simt", st,
-               (score_emit_simt<T><<<dim3(ceil_div(d.N, kEmitChunk), d.units), kEmitThreads, smem,
-                                     st>>>(d, Q, K, part, l.n_stat_chunks, a)));
+    const dim3 grid_s(l.n_stat_chunks, d.units), grid_e(ceil_div(d.N, kEmitChunk), d.units);
+    if (d.D == 64) {
+        GKV_LAUNCH("score_stats_simt", st,
+                   (score_stats_simt<T, 64><<<grid_s, threads, 0, st>>>(d, Q, K, part, l.n_stat_chunks,
+                                                                        at<int>(ws, l.status))));
+        GKV_LAUNCH("score_emit_simt", st,
+                   (score_emit_simt<T, 64><<<grid_e, kEmitThreads, smem, st>>>(d, Q, K, part, l.n_stat_chunks, a)));
+    } else {
+        GKV_LAUNCH("score_stats_simt", st,
+                   (score_stats_simt<T, 128><<<grid_s, threads, 0, st>>>(d, Q, K, part, l.n_stat_chunks,
+                                                                         at<int>(ws, l.status))));
+        GKV_LAUNCH("score_emit_simt", st,
+                   (score_emit_simt<T, 128><<<grid_e, kEmitThreads, smem, st>>>(d, Q, K, part, l.n_stat_chunks, a)));
+    }
     return launch_status();
 }
 
@@ -522,14 +533,14 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
 
 constexpr EmitExtras kPlainEmit{0, nullptr, nullptr, nullptr, 0, true};
 
-inline bool tc_mass(const __nv_bfloat16 *) { return !env_int("GRAPHKV_FORCE_SIMT", 0); }
-inline bool tc_mass(const float *) { return false; }
+inline bool tc_mass(const __nv_bfloat16 *, const Dims &d) { return d.D == kHeadDim && !env_int("GRAPHKV_FORCE_SIMT", 0); }
+inline bool tc_mass(const float *, const Dims &) { return false; }
 
 inline graphkv_status run_mass(const Dims &d, const Layout &l, const __nv_bfloat16 *Q,
                                const __nv_bfloat16 *K, float *a, void *ws, cudaStream_t st,
                                const EmitExtras &ex = kPlainEmit)
 {
-    if (!tc_mass(Q)) return run_mass_simt(d, l, Q, K, a, ws, st);
+    if (!tc_mass(Q, d)) return run_mass_simt(d, l, Q, K, a, ws, st);
     return run_mass_tc(d, l, Q, K, a, ws, st, ex);
 }
 inline graphkv_status run_mass(const Dims &d, const Layout &l, const float *Q, const float *K,
@@ -646,10 +657,14 @@ graphkv_status run_graph(const Dims &d, const Layout &l, const EdgeOperands<T> &
         return GRAPHKV_OK;
     }
     float *sims = at<float>(ws, l.sims);
-    GKV_LAUNCH("similarity_simt", st,
-               (similarity_simt<T><<<dim3(ceil_div(d.N, kSimChunk), d.units), kSimThreads, 0, st>>>(
-                   d, eo.S, Strides3{{eo.ss[0], eo.ss[1], eo.ss[2]}}, eo.A, Strides3{{eo.as[0], eo.as[1], eo.as[2]}},
-                   src, sims)));
+    const dim3 grid_sim(ceil_div(d.N, kSimChunk), d.units);
+    const Strides3 st_s{{eo.ss[0], eo.ss[1], eo.ss[2]}}, st_a{{eo.as[0], eo.as[1], eo.as[2]}};
+    if (d.D == 64)
+        GKV_LAUNCH("similarity_simt", st,
+                   (similarity_simt<T, 64><<<grid_sim, kSimThreads, 0, st>>>(d, eo.S, st_s, eo.A, st_a, src, sims)));
+    else
+        GKV_LAUNCH("similarity_simt", st,
+                   (similarity_simt<T, 128><<<grid_sim, kSimThreads, 0, st>>>(d, eo.S, st_s, eo.A, st_a, src, sims)));
     SelectArgs na{sims, d.N, d.N, d.m, src, at<int>(ws, l.nbr_idx), at<float>(ws, l.nbr_e)};
     GKV_LAUNCH("select_neighbors", st,
                (topk_select_kernel<<<d.units * d.K_src, kSelectThreads, 0, st>>>(na)));
@@ -721,7 +736,7 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const 
         SelectArgs sa{s, d.N, d.N, d.B, nullptr, idx_out, nullptr};
         GKV_LAUNCH("select_budget", st, (topk_select_kernel<<<d.units, kSelectThreads, 0, st>>>(sa)));
         if (K || V) {
-            const long long total = (long long)d.units * (d.B + d.W) * (kHeadDim * elem_bytes / 16);
+            const long long total = (long long)d.units * (d.B + d.W) * (d.D * elem_bytes / 16);
             const int blocks = (int)std::min<long long>((total + kGatherThreads - 1) / kGatherThreads,
                                                         148LL * 16);
             GKV_LAUNCH("gather_rows", st,
@@ -804,7 +819,7 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
     // (one sweep of at most 64 sources, one launch group, max pooling).  Measured on B200 the
     // merge in front of every similarity CTA costs what the pooling kernel takes (32K keys: 114
     // against 112 us per step; 131072 x 4: 1.25 against 1.13 ms), so it is off by default.
-    const bool tail_src = tc_mass(Q) && tc_graph && d.K_src <= tc::kSrcMaxK && !d.pool_avg &&
+    const bool tail_src = tc_mass(Q, d) && tc_graph && d.K_src <= tc::kSrcMaxK && !d.pool_avg &&
                           units_per_group(d) >= d.units && env_int("GRAPHKV_TAIL_SOURCES", 0);
     const bool finish_pools = d.kp > 1 && !d.pool_avg && (tail_src || !graph) && finish_plan(d, halo).ok &&
                               cluster_plan(d).ok;
@@ -821,7 +836,7 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
         if ((rc = run_mass(d, l, Q, K, a, ws, st)) != GRAPHKV_OK) return rc;
         // the tensor-core emit sweep leaves a histogram of the attention mass behind
         rc = run_pool_sources(d, d.kp > 1 ? a : nullptr, s, d.K_src, src,
-                              tc_mass(Q) ? at<uint32_t>(ws, l.a_hist) : nullptr,
+                              tc_mass(Q, d) ? at<uint32_t>(ws, l.a_hist) : nullptr,
                               tc_graph ? at<uint32_t>(ws, l.cand_hist) : nullptr, d.K_src * kCandBins, st);
         if (rc != GRAPHKV_OK) return rc;
     }
@@ -852,14 +867,15 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
 // ---- KNorm initial score ---------------------------------------------------------------------
 // s_j = 1 / max(||k_j||, eps) for the prefix keys: 16 threads share a key row (16 bytes each of a
 // bf16 row, 32 of an fp32 row), eight rows in flight per thread.  grid (CTAs per unit, units).
-template <typename T>
+template <typename T, int kD>
 __global__ void __launch_bounds__(256) knorm_score_kernel(Dims d, const T *__restrict__ K, float *__restrict__ scores)
 {
-    const int sub = threadIdx.x & 15, unit = blockIdx.y;
-    const T *Kh = K + (unit / d.hkv) * d.ks[0] + (long long)(unit % d.hkv) * d.ks[1] + sub * (kHeadDim / 16);
+    constexpr int kTpr = kD / 8;                 // threads per key row, eight elements each
+    const int sub = threadIdx.x & (kTpr - 1), unit = blockIdx.y;
+    const T *Kh = K + (unit / d.hkv) * d.ks[0] + (long long)(unit % d.hkv) * d.ks[1] + sub * 8;
     float *out = scores + (long long)unit * d.N;
-    const int stride = (gridDim.x * blockDim.x) >> 4;
-    for (int j0 = (blockIdx.x * blockDim.x + threadIdx.x) >> 4; j0 < d.N; j0 += 8 * stride) {
+    const int stride = (gridDim.x * blockDim.x) / kTpr;
+    for (int j0 = (blockIdx.x * blockDim.x + threadIdx.x) / kTpr; j0 < d.N; j0 += 8 * stride) {
         float n2[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -875,7 +891,7 @@ __global__ void __launch_bounds__(256) knorm_score_kernel(Dims d, const T *__res
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1) n2[u] += __shfl_xor_sync(0xffffffffu, n2[u], o);
+            for (int o = kTpr / 2; o > 0; o >>= 1) n2[u] += __shfl_xor_sync(0xffffffffu, n2[u], o);
             const int j = j0 + u * stride;
             if (sub == 0 && j < d.N) out[j] = 1.0f / fmaxf(sqrtf(n2[u]), kNormEps);
         }
@@ -1022,12 +1038,16 @@ graphkv_status graphkv_score_knorm(const graphkv_params *params, const void *K, 
     // about one wave of resident CTAs (eight of 256 threads per SM) over all units
     const int per_unit = std::max(1, std::min(ceil_div(d.N, 16 * 8), ceil_div(sm_count() * 8, d.units)));
     const dim3 grid(per_unit, d.units);
-    if (params->dtype == GRAPHKV_BF16)
-        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
-                                          d, static_cast<const __nv_bfloat16 *>(K), scores)));
+    const __nv_bfloat16 *Kb = static_cast<const __nv_bfloat16 *>(K);
+    const float *Kf = static_cast<const float *>(K);
+    if (params->dtype == GRAPHKV_BF16 && d.D == 64)
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<__nv_bfloat16, 64><<<grid, 256, 0, st>>>(d, Kb, scores)));
+    else if (params->dtype == GRAPHKV_BF16)
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(d, Kb, scores)));
+    else if (d.D == 64)
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<float, 64><<<grid, 256, 0, st>>>(d, Kf, scores)));
     else
-        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<float><<<grid, 256, 0, st>>>(
-                                          d, static_cast<const float *>(K), scores)));
+        GKV_LAUNCH("knorm_score", st, (knorm_score_kernel<float, 128><<<grid, 256, 0, st>>>(d, Kf, scores)));
     return launch_status();
 }
 

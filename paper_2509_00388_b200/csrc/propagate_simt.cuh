@@ -20,13 +20,13 @@ struct Strides3 {
     long long v[3];
 };
 
-template <typename T>
+template <typename T, int kD>
 __global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *__restrict__ S, Strides3 ss,
                                                              const T *__restrict__ K, Strides3 ks,
                                                              const int *__restrict__ src,
                                                              float *__restrict__ sims)
 {
-    __shared__ __align__(16) float srows[kMaxSrcSmem * kHeadDim];   // unit-norm source keys
+    __shared__ __align__(16) float srows[kMaxSrcSmem * kD];   // unit-norm source keys
     const int unit = blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
     const T *Kh = K + b * ks.v[0] + (long long)h * ks.v[1];
     const T *Sh = S + b * ss.v[0] + (long long)h * ss.v[1];
@@ -41,8 +41,10 @@ __global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *
         for (int a = warp; a < na; a += kSimThreads / 32) {
             const int i = src[(long long)unit * d.K_src + a0 + a];
             const T *kp = Sh + (long long)i * ss.v[2] + lane * 4;
-            float v[4];
-            if constexpr (sizeof(T) == 2) {
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            if (lane * 4 >= kD) {
+                // a row of 64 elements takes the first 16 lanes
+            } else if constexpr (sizeof(T) == 2) {
                 const uint2 raw = *reinterpret_cast<const uint2 *>(kp);
                 v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xffff0000u);
                 v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xffff0000u);
@@ -52,15 +54,16 @@ __global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *
             }
             const float n2 = warp_sum(v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3]);
             const float inv = 1.0f / fmaxf(sqrtf(n2), kNormEps);
-            *reinterpret_cast<float4 *>(srows + a * kHeadDim + lane * 4) =
-                make_float4(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv);
+            if (lane * 4 < kD)
+                *reinterpret_cast<float4 *>(srows + a * kD + lane * 4) =
+                    make_float4(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv);
         }
         __syncthreads();
         for (int j = j0 + threadIdx.x; j < j1; j += kSimThreads) {
-            float k[kHeadDim];
+            float k[kD];
             float n2 = 0.f;
 #pragma unroll
-            for (int c = 0; c < kHeadDim / 8; ++c) {
+            for (int c = 0; c < kD / 8; ++c) {
                 float v[8];
                 load8(Kh + (long long)j * ks.v[2] + c * 8, v);
 #pragma unroll
@@ -71,10 +74,10 @@ __global__ void __launch_bounds__(kSimThreads) similarity_simt(Dims d, const T *
             }
             const float inv = 1.0f / fmaxf(sqrtf(n2), kNormEps);
             for (int a = 0; a < na; ++a) {
-                const float4 *sv = reinterpret_cast<const float4 *>(srows + a * kHeadDim);
+                const float4 *sv = reinterpret_cast<const float4 *>(srows + a * kD);
                 float a0f = 0.f, a1f = 0.f, a2f = 0.f, a3f = 0.f;
 #pragma unroll
-                for (int c = 0; c < kHeadDim / 4; ++c) {
+                for (int c = 0; c < kD / 4; ++c) {
                     const float4 x = sv[c];
                     a0f = fmaf(x.x, k[4 * c], a0f);
                     a1f = fmaf(x.y, k[4 * c + 1], a1f);

@@ -1,5 +1,6 @@
 // Step (I), SIMT fp32 path: SnapKV-style window-attention scores for any input dtype.
-// Used for fp32 inputs (the tensor-core path takes bf16 only).  Two sweeps over the keys of a
+// Used for fp32 inputs and for a head dimension of 64 (the tensor-core path takes bf16 and 128
+// only); kD = 64 or 128.  Two sweeps over the keys of a
 // head: (1) per-row softmax statistics, (2) the column sums of the normalised probabilities.
 #pragma once
 
@@ -17,13 +18,13 @@ constexpr int kEmitChunk = 512;     // keys per CTA in the emit sweep
 // row r may see (prefix keys and window keys N + r' with r' <= r).
 // grid (n_chunks, units), block = GW rounded up to a warp multiple.
 // part [units][n_chunks][GW][2].
-template <typename T>
+template <typename T, int kD>
 __global__ void __launch_bounds__(kMaxRows) score_stats_simt(Dims d, const T *__restrict__ Q,
                                                             const T *__restrict__ K,
                                                             float *__restrict__ part,
                                                             int n_chunks, int *status_word)
 {
-    __shared__ __align__(16) float tile[kStatsTile * kHeadDim];
+    __shared__ __align__(16) float tile[kStatsTile * kD];
     const int unit = blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
     const int chunk = blockIdx.x;
     const int r = threadIdx.x;
@@ -31,12 +32,12 @@ __global__ void __launch_bounds__(kMaxRows) score_stats_simt(Dims d, const T *__
     const int g = active ? r / d.W : 0, rw = active ? r % d.W : 0;
     if (status_word && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status_word = 0;
 
-    float q[kHeadDim];
+    float q[kD];
     {
         const T *qp = Q + b * d.qs[0] + (long long)(h * d.G + g) * d.qs[1] + rw * d.qs[2];
-        const float scale = rsqrtf((float)kHeadDim) * kLog2e;
+        const float scale = rsqrtf((float)kD) * kLog2e;
 #pragma unroll
-        for (int c = 0; c < kHeadDim / 8; ++c) {
+        for (int c = 0; c < kD / 8; ++c) {
             float v[8];
             load8(qp + c * 8, v);
 #pragma unroll
@@ -51,11 +52,11 @@ __global__ void __launch_bounds__(kMaxRows) score_stats_simt(Dims d, const T *__
     for (int t0 = j0; t0 < j1; t0 += kStatsTile) {
         const int nt = min(kStatsTile, j1 - t0);
         __syncthreads();
-        for (int i = threadIdx.x; i < nt * (kHeadDim / 8); i += blockDim.x) {
-            const int kk = i / (kHeadDim / 8), c = i % (kHeadDim / 8);
+        for (int i = threadIdx.x; i < nt * (kD / 8); i += blockDim.x) {
+            const int kk = i / (kD / 8), c = i % (kD / 8);
             float v[8];
             load8(Kh + (long long)(t0 + kk) * d.ks[2] + c * 8, v);
-            float4 *dst = reinterpret_cast<float4 *>(tile + kk * kHeadDim + c * 8);
+            float4 *dst = reinterpret_cast<float4 *>(tile + kk * kD + c * 8);
             dst[0] = make_float4(v[0], v[1], v[2], v[3]);
             dst[1] = make_float4(v[4], v[5], v[6], v[7]);
         }
@@ -63,10 +64,10 @@ __global__ void __launch_bounds__(kMaxRows) score_stats_simt(Dims d, const T *__
         if (!active) continue;
         for (int kk = 0; kk < nt; ++kk) {
             if (t0 + kk > last_visible) break;
-            const float4 *kv = reinterpret_cast<const float4 *>(tile + kk * kHeadDim);
+            const float4 *kv = reinterpret_cast<const float4 *>(tile + kk * kD);
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
 #pragma unroll
-            for (int c = 0; c < kHeadDim / 4; ++c) {
+            for (int c = 0; c < kD / 4; ++c) {
                 const float4 x = kv[c];
                 acc0 = fmaf(q[4 * c], x.x, acc0);
                 acc1 = fmaf(q[4 * c + 1], x.y, acc1);
@@ -89,7 +90,7 @@ __global__ void __launch_bounds__(kMaxRows) score_stats_simt(Dims d, const T *__
 // Second sweep: a[j] = sum_r 2^(l2[r][j] - mx_r) / Z_r for the prefix keys j of one head.
 // grid (ceil(N / kEmitChunk), units), block kEmitThreads; dynamic shared memory holds the
 // scaled queries [GW][D] fp32 and the merged row statistics.
-template <typename T>
+template <typename T, int kD>
 __global__ void __launch_bounds__(kEmitThreads) score_emit_simt(Dims d, const T *__restrict__ Q,
                                                               const T *__restrict__ K,
                                                               const float *__restrict__ part,
@@ -98,19 +99,19 @@ __global__ void __launch_bounds__(kEmitThreads) score_emit_simt(Dims d, const T 
 {
     extern __shared__ __align__(16) float sm[];
     float *qs = sm;                         // [GW][D]
-    float *row_mx = sm + d.GW * kHeadDim;   // [GW]
+    float *row_mx = sm + d.GW * kD;   // [GW]
     float *row_w = row_mx + d.GW;           // [GW] = 1 / Z_r
     const int unit = blockIdx.y, b = unit / d.hkv, h = unit % d.hkv;
 
-    const float scale = rsqrtf((float)kHeadDim) * kLog2e;
-    for (int i = threadIdx.x; i < d.GW * (kHeadDim / 8); i += blockDim.x) {
-        const int r = i / (kHeadDim / 8), c = i % (kHeadDim / 8);
+    const float scale = rsqrtf((float)kD) * kLog2e;
+    for (int i = threadIdx.x; i < d.GW * (kD / 8); i += blockDim.x) {
+        const int r = i / (kD / 8), c = i % (kD / 8);
         const int g = r / d.W, rw = r % d.W;
         const T *qp = Q + b * d.qs[0] + (long long)(h * d.G + g) * d.qs[1] + rw * d.qs[2];
         float v[8];
         load8(qp + c * 8, v);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) qs[r * kHeadDim + c * 8 + e] = v[e] * scale;
+        for (int e = 0; e < 8; ++e) qs[r * kD + c * 8 + e] = v[e] * scale;
     }
     for (int r = threadIdx.x; r < d.GW; r += blockDim.x) {
         const float *p = part + ((long long)unit * n_chunks * d.GW + r) * 2;
@@ -128,9 +129,9 @@ __global__ void __launch_bounds__(kEmitThreads) score_emit_simt(Dims d, const T 
     const int j0 = blockIdx.x * kEmitChunk;
     const int j1 = min(j0 + kEmitChunk, d.N);
     for (int j = j0 + threadIdx.x; j < j1; j += kEmitThreads) {
-        float k[kHeadDim];
+        float k[kD];
 #pragma unroll
-        for (int c = 0; c < kHeadDim / 8; ++c) {
+        for (int c = 0; c < kD / 8; ++c) {
             float v[8];
             load8(Kh + (long long)j * d.ks[2] + c * 8, v);
 #pragma unroll
@@ -138,10 +139,10 @@ __global__ void __launch_bounds__(kEmitThreads) score_emit_simt(Dims d, const T 
         }
         float acc = 0.f;
         for (int r = 0; r < d.GW; ++r) {
-            const float4 *qv = reinterpret_cast<const float4 *>(qs + r * kHeadDim);
+            const float4 *qv = reinterpret_cast<const float4 *>(qs + r * kD);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-            for (int c = 0; c < kHeadDim / 4; ++c) {
+            for (int c = 0; c < kD / 4; ++c) {
                 const float4 x = qv[c];
                 a0 = fmaf(x.x, k[4 * c], a0);
                 a1 = fmaf(x.y, k[4 * c + 1], a1);

@@ -67,7 +67,7 @@ def test_invalid_params_are_rejected_on_the_host(bad):
 
 def test_unsupported_shapes():
     p = _params()
-    p.head_dim = 64
+    p.head_dim = 96                                       # 128 and 64 are served
     assert gk.lib().graphkv_score(C.byref(p), 16, 16, 16, 256, 1 << 30, None) == gk.ERR_UNSUPPORTED
     p = _params()
     p.n_q_heads, p.window, p.seq_len = 64, 64, 164      # G*W = 2048 rows

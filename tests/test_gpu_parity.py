@@ -264,6 +264,14 @@ def test_one_score_kernel_and_two_agree_to_the_bit(gk, window):
     want = okv.score(inp["Qw"], inp["K"], cfg.window, cfg.pool_kernel)
     assert pu.score_rel_err(one.cpu(), want) <= pu.SCORE_RTOL
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_head_dimension_64(gk, dtype):
+    # heads of 64 dimensions take the general kernels for the scores, the edges and the gather
+    # (the tensor-core kernels are written for 128) and the same row kernels
+    cfg = wl.scaled(wl.LLAMA_32K, head_dim=64, dtype=dtype, n_prefix=3000 + 21, budget=200, n_q_heads=8,
+                    n_kv_heads=2, n_clusters=24, neighbors=8, batch=2)
+    check(gk, cfg, strict_overlap=False)
+
 
 @pytest.mark.parametrize("case", [
     dict(topk_nodes=40, neighbors=12),                  # source count padded to 64

@@ -34,9 +34,11 @@ def kwargs(cfg, **extra):
     return d
 
 
+@pytest.mark.parametrize("head_dim", [128, 64])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
-def test_knorm_scores_and_the_path_behind_them(gk, dtype):
-    cfg = small_cfg(dtype=dtype, n_prefix=4500 if dtype == "bf16" else 1800)
+def test_knorm_scores_and_the_path_behind_them(gk, dtype, head_dim):
+    cfg = small_cfg(dtype=dtype, head_dim=head_dim,
+                    n_prefix=4500 if dtype == "bf16" and head_dim == 128 else 1800)
     inp = wl.make_inputs(cfg)
     Kd, Vd = inp["K"].to(DEV), inp["V"].to(DEV)
     kw = kwargs(cfg)
