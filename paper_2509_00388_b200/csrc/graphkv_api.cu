@@ -201,7 +201,13 @@ SimPlan sim_plan(const Dims &d, bool bf16)
         return p;
     if (env_int("GRAPHKV_FORCE_SIMT", 0)) return p;
     if (!cluster_plan(d).ok) return p;          // its candidate lists are merged by the cluster kernel
-    p.NP = d.K_src <= 16 ? 16 : (d.K_src <= 32 ? 32 : 64);
+    // 64 sources per sweep leave a CTA 8 key tiles (the tensor memory holds 512 columns): four keys per
+    // epilogue thread, of which the m + 1 best maxima set each source's threshold.  With more than 16
+    // neighbours the chunk's candidates then crowd its 64-entry lists and the threads' queues, and
+    // overflows take the slow exact path (450 sources, m = 32 at 32K keys: 2.1 ms against 0.35 ms);
+    // 32 sources per sweep (16 tiles, eight keys per thread) stay clear of it and measured faster
+    // there at every source count, 64 faster for m = 16.
+    p.NP = d.K_src <= 16 ? 16 : (d.K_src <= 32 || d.m > 16 ? 32 : 64);
     p.stages = p.NP == 64 ? 4 : 5;
     const int cap = 512 / p.NP;
     const int group = units_per_group(d);
