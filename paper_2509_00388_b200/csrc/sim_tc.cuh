@@ -13,7 +13,7 @@
 //   2. re-reads TMEM and lists the edges whose bin (the same expression as in step 1, so that a
 //      counted maximum is always listed) reaches it, excluding the source itself;
 //   3. if a list outgrows its capacity (many ties), finds that source's exact m-th largest
-//      (edge descending, position ascending) by bisection over counting passes and lists
+//      (edge descending, position ascending) by a byte-wise radix search over TMEM and lists
 //      exactly those m.
 // The lists of all chunks hold every member of the head-wide top-m.  Each listed edge is also
 // counted in a per-source histogram over the cosine, from which the row-wise finishing kernel
@@ -451,24 +451,74 @@ similarity_tc(const __grid_constant__ CUtensorMap tmK, SimTcArgs a)
             asm volatile("bar.sync 1, 256;" ::: "memory");
             for (int c = 0; c < n_src && any_overflow; ++c) {
                 if (cnt[c] <= kCandCap) continue;                 // uniform: shared memory value
+                // the m-th largest 64-bit edge key of the chunk (keys are distinct: distinct positions),
+                // a byte at a time from the top: a 256-bin histogram of the byte among the keys that
+                // share the bytes found so far, the digit that holds the m-th largest, eight rounds
                 unsigned long long t64 = 0ull;
                 const float sinv = src_inv[c];
                 const int self = src_pos[c];
-                for (int bit = 63; bit >= 0; --bit) {
-                    const unsigned long long cand = t64 | (1ull << bit);
-                    int n = 0;
+                uint32_t *rh = max_bin;                           // [256] (the stage memory is idle)
+                uint32_t remaining = (uint32_t)d.m;
+                for (int byte = 7; byte >= 0; --byte) {
+                    const unsigned long long hi_mask = byte == 7 ? 0ull : ~0ull << (8 * (byte + 1));
+                    rh[et] = 0u;
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
                     for (int i = set; i < n_local; i += 2) {
                         const int j = (t0 + i) * kTileKeys + key_lane;
                         const float dot = tmem_ld1(lane_addr + i * NP + c);
                         const float e = fminf(fmaxf(dot * inv_norm[i * 128 + key_lane] * sinv, -1.0f), 1.0f);
-                        n += (j < d.N && j != self && edge_key(e, j) >= cand) ? 1 : 0;
+                        const unsigned long long key = edge_key(e, j);
+                        const bool valid = j < d.N && j != self && (key & hi_mask) == t64;
+                        const uint32_t bin = (uint32_t)(key >> (8 * byte)) & 0xffu;
+                        // (cosines of a chunk crowd into few digits: the lanes that share the first
+                        // valid lane's digit are counted with one addition)
+                        const unsigned vm = __ballot_sync(0xffffffffu, valid);
+                        if (vm) {
+                            const int leader = __ffs(vm) - 1;
+                            const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
+                            const bool same = valid && bin == lbin;
+                            const unsigned sm = __ballot_sync(0xffffffffu, same);
+                            if (lane == leader) atomicAdd(&rh[lbin], (uint32_t)__popc(sm));
+                            else if (valid && !same) atomicAdd(&rh[bin], 1u);
+                        }
                     }
-                    n = __reduce_add_sync(0xffffffffu, n);
-                    if (et == 0) xchg[bit & 1] = 0;
                     asm volatile("bar.sync 1, 256;" ::: "memory");
-                    if (lane == 0 && n) atomicAdd(&xchg[bit & 1], n);
+                    if (warp == 2) {
+                        // lane l holds digits 255 - 8 l - q (q < 8): counts above each digit by a scan
+                        uint32_t c8[8], sum = 0;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            c8[q] = rh[255 - 8 * lane - q];
+                            sum += c8[q];
+                        }
+                        uint32_t incl = sum;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                            if (lane >= o) incl += t;
+                        }
+                        const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+                        uint32_t run = incl - sum;
+                        if (lane == 0) {
+                            xchg[0] = 0;                            // fewer keys than m: every key is kept
+                            xchg[1] = (int)remaining;
+                        }
+                        __syncwarp();
+                        if (total >= remaining) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                if (run < remaining && run + c8[q] >= remaining) {
+                                    xchg[0] = 255 - 8 * lane - q;
+                                    xchg[1] = (int)(remaining - run);
+                                }
+                                run += c8[q];
+                            }
+                        }
+                    }
                     asm volatile("bar.sync 1, 256;" ::: "memory");
-                    if (xchg[bit & 1] >= d.m) t64 = cand;
+                    t64 |= (unsigned long long)(uint32_t)xchg[0] << (8 * byte);
+                    remaining = (uint32_t)xchg[1];
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
                 }
                 if (et == 0) cnt[c] = 0;
                 asm volatile("bar.sync 1, 256;" ::: "memory");
