@@ -570,45 +570,101 @@ __device__ __forceinline__ void cluster_emit_sorted(cg::cluster_group &cl, int C
 }
 
 // The m largest edges (cosine descending, position ascending) of the lists when too many tie at
-// the bound: exact m-th largest by bisection over the lists themselves.  One warp; returns the
-// number of survivors written (m, or fewer when fewer edges are listed).
-__device__ int merge_exact(const Cand *cand, int slots, int m, Cand *surv)
+// the bound: the exact m-th largest 64-bit edge key (keys are distinct: distinct positions) by a
+// byte-wise radix search over the lists themselves, eight rounds of a 256-bin histogram of the byte
+// among the keys that share the bytes found so far.  The four warps of a merging group (`wg` of
+// them, barrier `bar_id`); `rh`: 264 words of shared memory of the group; the number of survivors
+// written (m, or fewer when fewer edges are listed) is left in *ns_sh.
+__device__ void merge_exact(const Cand *cand, int slots, int m, Cand *surv, uint32_t *rh, int *ns_sh,
+                            int bar_id, int wg)
 {
-    const int lane = threadIdx.x & 31;
-    int ns = 0;
-    {
-        // too many ties at the bound: exact m-th largest by bisection over the lists themselves
-        unsigned long long t64 = 0ull;
-        for (int bit = 63; bit >= 0; --bit) {
-            const unsigned long long cut = t64 | (1ull << bit);
-            int n = 0;
-            for (int i = lane; i < slots; i += 32) {
-                const unsigned long long raw = __ldcg(reinterpret_cast<const unsigned long long *>(cand + i));
-                const float e = __uint_as_float(static_cast<uint32_t>(raw));
-                n += e >= -1.0f && edge_key(e, static_cast<int>(raw >> 32)) >= cut;
-            }
-            n = __reduce_add_sync(0xffffffffu, n);
-            if (n >= m) t64 = cut;
-        }
-        ns = 0;
-        for (int i0 = 0; i0 < slots; i0 += 32) {
-            const int i = i0 + lane;
-            bool keep = false;
-            Cand cd{0.f, 0};
+    const int lane = threadIdx.x & 31, t = wg * 32 + lane;
+    unsigned long long t64 = 0ull;
+    uint32_t remaining = (uint32_t)m;
+    for (int byte = 7; byte >= 0; --byte) {
+        const unsigned long long hi_mask = byte == 7 ? 0ull : ~0ull << (8 * (byte + 1));
+        rh[t] = 0u;
+        rh[t + 128] = 0u;
+        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+        for (int i0 = 0; i0 < slots; i0 += 128) {
+            const int i = i0 + t;
+            bool valid = false;
+            uint32_t bin = 0;
             if (i < slots) {
                 const unsigned long long raw = __ldcg(reinterpret_cast<const unsigned long long *>(cand + i));
-                cd.e = __uint_as_float(static_cast<uint32_t>(raw));
-                cd.j = static_cast<int>(raw >> 32);
-                keep = cd.e >= -1.0f && edge_key(cd.e, cd.j) >= t64;
+                const float e = __uint_as_float(static_cast<uint32_t>(raw));
+                const unsigned long long key = edge_key(e, static_cast<int>(raw >> 32));
+                valid = e >= -1.0f && (key & hi_mask) == t64;
+                bin = (uint32_t)(key >> (8 * byte)) & 0xffu;
             }
-            const unsigned bm = __ballot_sync(0xffffffffu, keep);
-            const int pos = ns + __popc(bm & ((1u << lane) - 1u));
+            // tied cosines share their digits: one addition for the lanes with the first valid lane's
+            const unsigned vm = __ballot_sync(0xffffffffu, valid);
+            if (vm) {
+                const int leader = __ffs(vm) - 1;
+                const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
+                const bool same = valid && bin == lbin;
+                const unsigned sm = __ballot_sync(0xffffffffu, same);
+                if (lane == leader) atomicAdd(&rh[lbin], (uint32_t)__popc(sm));
+                else if (valid && !same) atomicAdd(&rh[bin], 1u);
+            }
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+        if (wg == 0) {
+            // lane l holds digits 255 - 8 l - q (q < 8)
+            uint32_t c8[8], sum = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                c8[q] = rh[255 - 8 * lane - q];
+                sum += c8[q];
+            }
+            const uint32_t incl = warp_incl_scan(sum, lane);
+            const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+            uint32_t run = incl - sum;
+            if (lane == 0) {
+                rh[256] = 0u;                               // fewer edges than m: all are kept
+                rh[257] = remaining;
+            }
+            __syncwarp();
+            if (total >= remaining) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (run < remaining && run + c8[q] >= remaining) {
+                        rh[256] = (uint32_t)(255 - 8 * lane - q);
+                        rh[257] = remaining - run;
+                    }
+                    run += c8[q];
+                }
+            }
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+        t64 |= (unsigned long long)rh[256] << (8 * byte);
+        remaining = rh[257];
+        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    }
+    if (t == 0) *ns_sh = 0;
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    for (int i0 = 0; i0 < slots; i0 += 128) {
+        const int i = i0 + t;
+        bool keep = false;
+        Cand cd{0.f, 0};
+        if (i < slots) {
+            const unsigned long long raw = __ldcg(reinterpret_cast<const unsigned long long *>(cand + i));
+            cd.e = __uint_as_float(static_cast<uint32_t>(raw));
+            cd.j = static_cast<int>(raw >> 32);
+            keep = cd.e >= -1.0f && edge_key(cd.e, cd.j) >= t64;
+        }
+        const unsigned bm = __ballot_sync(0xffffffffu, keep);
+        if (bm) {
+            int basep = 0;
+            if (lane == 0) basep = atomicAdd(ns_sh, __popc(bm));
+            basep = __shfl_sync(0xffffffffu, basep, 0);
+            const int pos = basep + __popc(bm & ((1u << lane) - 1u));
             if (keep && pos < kSurvCap) surv[pos] = cd;
-            ns += __popc(bm);
         }
     }
-    __syncwarp();
-    return min(ns, kSurvCap);
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    if (t == 0) *ns_sh = min(*ns_sh, kSurvCap);
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
 }
 
 // Eq. 3 for one source: the m largest edges (cosine descending, position ascending) among the
@@ -632,7 +688,7 @@ struct PushLists {
 
 __device__ void merge_neighbours(cg::cluster_group &cl, const Cand *cand, const uint32_t *hist,
                                  int chunks, int m, Cand *surv, int *ns_sh, int bar_id, int wg,
-                                 int *nbr_idx, float *nbr_e, const PushLists &push)
+                                 int *nbr_idx, float *nbr_e, const PushLists &push, uint32_t *rh)
 {
     const int lane = threadIdx.x & 31;
     constexpr int kPer = kCandBins / 32;
@@ -709,9 +765,7 @@ __device__ void merge_neighbours(cg::cluster_group &cl, const Cand *cand, const 
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
     int ns = *ns_sh;
     if (ns > kSurvCap) {
-        if (wg == 0) ns = merge_exact(cand, slots, m, surv);
-        if (wg == 0 && lane == 0) *ns_sh = ns;
-        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+        merge_exact(cand, slots, m, surv, rh, ns_sh, bar_id, wg);
         ns = *ns_sh;
     }
     // rank by counting: all keys are distinct (distinct positions)
@@ -1266,7 +1320,7 @@ __global__ void __launch_bounds__(kThreads, 1) finish_kernel(FinishArgs a)
                 merge_neighbours(cl, a.cand + slot * kCandCap,
                                  a.cand_hist + ((long long)unit * d.K_src + src) * kCandBins,
                                  a.cand_chunks, d.m, surv, ns_sh, 1 + grp, wg, ni + src * d.m,
-                                 ne + src * d.m, push);
+                                 ne + src * d.m, push, s.fine + grp * 264);
             }
             pc.mark();
             if (!staged) __threadfence();                     // the lists are read back from global memory
