@@ -1,6 +1,7 @@
 // C ABI of the GraphKV library: argument validation, workspace layout and kernel launches.
 #include <algorithm>
 #include <atomic>
+#include <chrono>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -383,12 +384,33 @@ template <typename Kern> bool set_smem(Kern k, size_t bytes)
     return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
 }
 
+// A value for the arrival words of the kernel of both score sweeps that no earlier call of this
+// process has used (never zero; the sequence starts at a clock-derived value, so a word left by
+// another process matches it only by a 1 in 2^32 chance).
+uint32_t next_call_tag()
+{
+    static std::atomic<uint32_t> tag{
+        static_cast<uint32_t>(std::chrono::steady_clock::now().time_since_epoch().count() * 2654435761u) | 1u};
+    uint32_t t = tag.fetch_add(1u) + 1u;
+    if (t == 0u) t = tag.fetch_add(1u) + 1u;
+    return t;
+}
+
+// Status word, arrival counters and the mass histogram start every scoring call at zero: a memset
+// ahead of the sweeps, except where the kernel of both sweeps clears them itself.
+inline graphkv_status reset_words(const Dims &d, const Layout &l, void *ws, cudaStream_t st)
+{
+    return cudaMemsetAsync(ws, 0, l.a_hist + (size_t)d.units * tc::kMassBins * sizeof(uint32_t), st) == cudaSuccess
+               ? GRAPHKV_OK : GRAPHKV_ERR_CUDA;
+}
+
 // ---- step (I) ------------------------------------------------------------------------------
 // Attention mass before pooling, a [units][N], SIMT path (any dtype).
 template <typename T>
 graphkv_status run_mass_simt(const Dims &d, const Layout &l, const T *Q, const T *K, float *a,
                              void *ws, cudaStream_t st)
 {
+    if (reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
     float *part = at<float>(ws, l.part);
     const int threads = ceil_div(d.GW, 32) * 32;
     const size_t smem = ((size_t)d.GW * d.D + 2 * d.GW) * sizeof(float);
@@ -492,6 +514,12 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
     const int tiles_stats = ceil_div(d.L, tc::kTileKeys), tiles_emit = ceil_div(d.N, tc::kTileKeys);
     const int group = units_per_group(d);
     graphkv_status rc = GRAPHKV_OK;
+    // the kernel of both sweeps (one launch of all units, all CTAs resident) clears the head of the
+    // workspace itself; every other form gets a memset first
+    const bool one_kernel = ex.k == 0 && group >= d.units &&
+                            d.units * sweep_chunks(d.units, tiles_stats, 1, l.max_parts) <= sm_count() &&
+                            !env_int("GRAPHKV_TWO_SCORE_KERNELS", 0);
+    if (!one_kernel && reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
     for (int u0 = 0; u0 < d.units && rc == GRAPHKV_OK; u0 += group) {
         const int nu = std::min(group, d.units - u0);
         const int chunks_s = sweep_chunks(nu, tiles_stats, 1, l.max_parts);
@@ -500,7 +528,7 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
                            ex.global_hist ? at<uint32_t>(ws, l.a_hist) : nullptr, at<int>(ws, l.status), u0,
                            chunks_s, tiles_stats, chunks_s, stages, 0,
                            tc::SourceArgs{0, 0, nullptr, nullptr, nullptr, 0, 0}, nullptr, 0, 0,
-                           wait_cycles(), env_int("GRAPHKV_DEBUG_WITHHOLD_COMMIT", 0)};
+                           wait_cycles(), 0, 0u, env_int("GRAPHKV_DEBUG_WITHHOLD_COMMIT", 0)};
         tc::ScoreTcArgs ea = sa;
         ea.chunks = chunks_e;
         ea.n_tiles = tiles_emit;
@@ -514,16 +542,19 @@ graphkv_status run_mass_tc(const Dims &d, const Layout &l, const __nv_bfloat16 *
         // of a unit wait for one another between the passes, so the launch is a cooperative one
         // (the device starts the grid only when all of it fits beside whatever else is running);
         // a device that refuses it gets the two kernels
-        if (ex.k == 0 && nu * chunks_s <= sm_count() && !env_int("GRAPHKV_TWO_SCORE_KERNELS", 0)) {
+        if (one_kernel) {
             tc::ScoreTcArgs fa = ea;
             fa.chunks = chunks_s;
             fa.n_tiles = tiles_stats;
+            fa.clear_head = 1;
+            fa.call_tag = next_call_tag();
             fa.wait_prior = next_launch_is_dependent();
             t_cooperative = true;
             rc = launch_ex("score_fused_tc", row_tiles == 1 ? tc::score_fused_tc<1> : tc::score_fused_tc<2>,
                            dim3(chunks_s, nu), dim3(tc::kScoreThreads), smem, st, fa.wait_prior != 0, 1, tmK, fa);
             if (rc == GRAPHKV_OK) continue;
             cudaGetLastError();
+            if (reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
             rc = GRAPHKV_OK;
         }
         sa.wait_prior = next_launch_is_dependent();
@@ -756,18 +787,11 @@ graphkv_status run_finish(const Dims &d, const Layout &l, int elem_bytes, const 
 }
 
 // ---- the calls, typed ---------------------------------------------------------------------------
-// Status word, arrival counters and the mass histogram start every scoring call at zero.
-inline graphkv_status reset_words(const Dims &d, const Layout &l, void *ws, cudaStream_t st)
-{
-    return cudaMemsetAsync(ws, 0, l.a_hist + (size_t)d.units * tc::kMassBins * sizeof(uint32_t), st) == cudaSuccess
-               ? GRAPHKV_OK : GRAPHKV_ERR_CUDA;
-}
 
 template <typename T>
 graphkv_status do_score(const Dims &d, const Layout &l, const T *Q, const T *K, float *scores,
                         void *ws, cudaStream_t st)
 {
-    if (reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
     float *a = d.kp > 1 ? at<float>(ws, l.a) : scores;
     graphkv_status rc = run_mass(d, l, Q, K, a, ws, st);
     if (rc != GRAPHKV_OK || d.kp == 1) return rc;
@@ -815,7 +839,6 @@ graphkv_status do_compress(const Dims &d, const Layout &l, const T *Q, const T *
                            cudaStream_t st)
 {
     const bool graph = graph_active(d);
-    if (reset_words(d, l, ws, st) != GRAPHKV_OK) return GRAPHKV_ERR_CUDA;
     float *a = d.kp > 1 ? at<float>(ws, l.a) : s;
     int *src = at<int>(ws, l.src);
     const bool tc_graph = graph && sim_plan(d, sizeof(T) == 2).ok;

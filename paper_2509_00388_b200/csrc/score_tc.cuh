@@ -37,9 +37,9 @@ struct ScoreTcArgs {
     const __nv_bfloat16 *Q;
     float *part;        // [units][stats_chunks][GW][2] row statistics (max, sum) per key chunk
     float *row_c;       // [units][GW] c_r = max_r + log2(Z_r), written by the last stats CTA of a unit
-    int *arrivals;      // [2 * units] counters of CTAs per unit (zero before the launch; reset on the way):
-                        // the two-kernel path counts finished statistics CTAs in [unit], the kernel of
-                        // both sweeps arrivals and departures of its hand-over in [2 * unit], [2 * unit + 1]
+    int *arrivals;      // [2 * units] words: the two-kernel path counts finished statistics CTAs in [unit]
+                        // (zero before the launch; reset on the way), the kernel of both sweeps keeps a
+                        // 64-bit (tag, count) word per unit there
     float *a_out;       // [units][N] attention mass before pooling
     uint32_t *a_hist;   // optional [units][kMassBins]: counts of a by the top bits of its ordered image
     int *status;        // workspace status word
@@ -56,6 +56,9 @@ struct ScoreTcArgs {
     int zero_words;
     int local_hist;     // build the per-CTA mass histogram even without a_hist
     long long wait_cycles;   // limit of every wait of the kernel, in clocks
+    int clear_head;          // kernel of both sweeps: clear the status word and the unit's mass histogram on
+                             // the way (the caller then needs no memset ahead of the launch)
+    uint32_t call_tag;       // kernel of both sweeps: a nonzero value no earlier call on this workspace used
     int withhold_commit;     // test hook (statistics sweep): 1: the MMA issuer leaves out the arrival that
                              // announces its first accumulator, so the wait for it runs out; 2 (kernel of
                              // both sweeps): no CTA announces itself at the hand-over, so that wait runs out
@@ -572,8 +575,8 @@ score_emit_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
 // pass left in the stage ring are used again without a copy.  Against two launches this saves a
 // kernel boundary, the second set-up (barriers, tensor memory, the staging of the queries) and
 // the re-read of the ring's tiles.  kTiles = 1 (G*W <= 128) or 2 (G*W <= 256); grid (chunks,
-// units of the launch); a.arrivals holds two counters per unit (arrived, departed), zero before
-// the launch and zero again after it.
+// units of the launch); a.arrivals holds one 64-bit word per unit (the call's tag and the count of
+// arrived CTAs), whatever its content before the launch.
 template <int kTiles>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_fused_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
@@ -625,6 +628,16 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     const bool want_hist = a.a_hist != nullptr || a.local_hist;
     if (want_hist)
         for (int i = threadIdx.x; i < kMassBins; i += kScoreThreads) mass_hist[i] = 0u;
+    if (a.clear_head) {
+        // (after the wait: nothing of the call before still reads or writes these words; the unit's
+        // histogram is added to only after the hand-over, which orders these stores before it)
+        if (a.status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *a.status = 0;
+        if (a.a_hist) {
+            const int per_cta = ceil_div(kMassBins, a.chunks);
+            for (int i = chunk * per_cta + threadIdx.x; i < min((chunk + 1) * per_cta, kMassBins); i += kScoreThreads)
+                a.a_hist[(long long)unit * kMassBins + i] = 0u;
+        }
+    }
     if (a.zero) {
         const int per_cta = ceil_div(a.zero_words, a.chunks);
         for (int i = chunk * per_cta + threadIdx.x; i < min((chunk + 1) * per_cta, a.zero_words); i += kScoreThreads)
@@ -725,15 +738,27 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
-        // a CTA whose pass failed still arrives, so that the others do not wait for it in vain
-        int *arrived = a.arrivals + 2 * unit;
-        if (a.withhold_commit != 2) atomicAdd(arrived, 1);
+        // The unit's arrival word holds (call tag, count).  A CTA that finds another tag there starts
+        // the count for this call, so whatever the word held before (zeros, an earlier call's count,
+        // the count of a call that gave up, memory nobody cleared) never counts: nothing has to be
+        // reset.  A CTA whose pass failed still arrives, so that the others do not wait in vain.
+        unsigned long long *arrived = reinterpret_cast<unsigned long long *>(a.arrivals) + unit;
+        const unsigned long long tag = (unsigned long long)a.call_tag << 32;
+        if (a.withhold_commit != 2) {
+            unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(arrived);
+            while (true) {
+                const unsigned long long nv = (old >> 32) == a.call_tag ? old + 1ull : (tag | 1ull);
+                const unsigned long long prev = atomicCAS(arrived, old, nv);
+                if (prev == old) break;
+                old = prev;
+            }
+        }
         bool in = false;
         const long long c0 = clock64();
         while (true) {
-            int seen;
-            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(arrived) : "memory");
-            if (seen >= a.chunks) { in = true; break; }
+            unsigned long long seen;
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(arrived) : "memory");
+            if ((seen >> 32) == a.call_tag && (uint32_t)seen >= (uint32_t)a.chunks) { in = true; break; }
             if (clock64() - c0 > lim) break;
             __nanosleep(20);
         }
@@ -755,14 +780,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        // the last CTA of the unit to leave the hand-over clears both counters for the next launch
-        int *cnt = a.arrivals + 2 * unit;
-        if (atomicAdd(cnt + 1, 1) == a.chunks - 1) {
-            atomicExch(cnt, 0);
-            atomicExch(cnt + 1, 0);
-        }
-    }
     pc.mark();
 
     // ---- emit pass: D = K Q^T, the chunk's prefix tiles in reverse order ----
