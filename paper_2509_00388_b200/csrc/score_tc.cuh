@@ -721,6 +721,10 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     // ---- hand-over: partials out, every chunk of the unit in, row constants ----
     tc_fence_before();
     bool all_ok = __syncthreads_and(ok ? 1 : 0) != 0;
+    unsigned long long *arrived = reinterpret_cast<unsigned long long *>(a.arrivals) + unit;
+    unsigned long long seen_early = 0ull;
+    if (threadIdx.x == 0)
+        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(seen_early) : "l"(arrived) : "memory");
     for (int r = threadIdx.x; r < d.GW; r += kScoreThreads) {
         float2 p[kParts];
         float mx = kNegBig;
@@ -739,18 +743,23 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmK, ScoreTcArgs a)
     __syncthreads();
     if (threadIdx.x == 0) {
         // The unit's arrival word holds (call tag, count).  A CTA that finds another tag there starts
-        // the count for this call, so whatever the word held before (zeros, an earlier call's count,
-        // the count of a call that gave up, memory nobody cleared) never counts: nothing has to be
-        // reset.  A CTA whose pass failed still arrives, so that the others do not wait in vain.
-        unsigned long long *arrived = reinterpret_cast<unsigned long long *>(a.arrivals) + unit;
+        // the count for this call (one compare-and-swap, by the unit's first arrivals only), so
+        // whatever the word held before (zeros, an earlier call's count, the count of a call that
+        // gave up, memory nobody cleared) never counts and nothing has to be reset; with the call's
+        // tag in place an arrival is a plain addition.  The word was looked at ahead of the fence
+        // (`seen_early`): its tag can only have turned into this call's since.  A CTA whose pass
+        // failed still arrives, so that the others do not wait in vain.
         const unsigned long long tag = (unsigned long long)a.call_tag << 32;
         if (a.withhold_commit != 2) {
-            unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(arrived);
+            unsigned long long cur = seen_early;
             while (true) {
-                const unsigned long long nv = (old >> 32) == a.call_tag ? old + 1ull : (tag | 1ull);
-                const unsigned long long prev = atomicCAS(arrived, old, nv);
-                if (prev == old) break;
-                old = prev;
+                if ((cur >> 32) == a.call_tag) {
+                    atomicAdd(arrived, 1ull);
+                    break;
+                }
+                const unsigned long long prev = atomicCAS(arrived, cur, tag | 1ull);
+                if (prev == cur) break;
+                cur = prev;
             }
         }
         bool in = false;
