@@ -28,10 +28,10 @@
  *   - Every top-k keeps exactly k items; equal values are ordered lower index first, so results
  *     are deterministic.
  *   - One workspace serves one call at a time: calls sharing a workspace must be ordered on
- *     one stream.  graphkv_score and graphkv_compress clear the status word at its head; a
- *     workspace whose first use is another call (graphkv_propagate after graphkv_score_knorm,
- *     graphkv_select_gather alone) must be zero-filled once by its owner for graphkv_read_status
- *     to mean anything.
+ *     one stream.  graphkv_score and graphkv_compress set up every word of it they rely on
+ *     (the status word at its head included), whatever it held before; a workspace whose first
+ *     use is another call (graphkv_propagate after graphkv_score_knorm, graphkv_select_gather
+ *     alone) must be zero-filled once by its owner for graphkv_read_status to mean anything.
  */
 #ifndef GRAPHKV_H_
 #define GRAPHKV_H_
