@@ -150,9 +150,16 @@ __device__ Threshold cluster_kth_t(cg::cluster_group &cl, int C, int rank, const
             const int slice = kBins / C;
             if (tid < slice) {
                 const int bin = rank * slice + tid;
+                // (all peers' counts requested before any is added: one round trip, not C)
+                uint32_t part[kMaxCluster];
+#pragma unroll
+                for (int p = 0; p < kMaxCluster; ++p) part[p] = p < C ? cl.map_shared_rank(s.hist, p)[bin] : 0u;
                 uint32_t sum = 0;
-                for (int p = 0; p < C; ++p) sum += cl.map_shared_rank(s.hist, p)[bin];
-                for (int p = 0; p < C; ++p) cl.map_shared_rank(s.tot, p)[bin] = sum;
+#pragma unroll
+                for (int p = 0; p < kMaxCluster; ++p) sum += part[p];
+#pragma unroll
+                for (int p = 0; p < kMaxCluster; ++p)
+                    if (p < C) cl.map_shared_rank(s.tot, p)[bin] = sum;
             }
             cl.sync();                                   // every CTA's copy of the totals is complete
             total = s.tot;
@@ -319,8 +326,13 @@ __device__ Threshold cluster_kth_fine_t(cg::cluster_group &cl, int C, int rank, 
     if (C > 1) {
         cl.sync();                                       // every CTA's histogram is complete
         for (int b = tid; b < slice; b += kThreads) {
+            uint32_t part[kMaxCluster];
+#pragma unroll
+            for (int p = 0; p < kMaxCluster; ++p)
+                part[p] = p < C ? cl.map_shared_rank(s.fine, p)[rank * slice + b] : 0u;
             uint32_t sum = 0;
-            for (int p = 0; p < C; ++p) sum += cl.map_shared_rank(s.fine, p)[rank * slice + b];
+#pragma unroll
+            for (int p = 0; p < kMaxCluster; ++p) sum += part[p];
             s.tot[b] = sum;
             mine += sum;
         }
