@@ -131,16 +131,12 @@ __device__ Threshold cluster_kth_t(cg::cluster_group &cl, int C, int rank, const
                 valid = (u & th.mask) == th.prefix;
                 bin = (u >> shift) & (nb - 1u);
             }
-            // lanes sharing the first valid lane's digit are counted with one atomic (scores of a
-            // row often crowd into one digit); the others add for themselves
+            // the lanes of a warp that share a digit are counted with one addition by the first of
+            // them (scores of a row crowd into few digits: additions to one word serialise)
             const unsigned vm = __ballot_sync(0xffffffffu, valid);
-            if (vm) {
-                const int leader = __ffs(vm) - 1;
-                const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
-                const bool same = valid && bin == lbin;
-                const unsigned sm = __ballot_sync(0xffffffffu, same);
-                if (lane == leader) atomicAdd(&s.hist[lbin], (uint32_t)__popc(sm));
-                else if (valid && !same) atomicAdd(&s.hist[bin], 1u);
+            if (valid) {
+                const unsigned peers = __match_any_sync(vm, bin);
+                if (lane == __ffs(peers) - 1) atomicAdd(&s.hist[bin], (uint32_t)__popc(peers));
             }
         }
         __syncthreads();
@@ -306,16 +302,11 @@ __device__ Threshold cluster_kth_fine_t(cg::cluster_group &cl, int C, int rank, 
         const int i = i0 + tid;
         const bool valid = i < n_local;
         const uint32_t bin = valid ? float_to_key(row.at<kListed>(i)) >> kFineShift : 0u;
-        // lanes sharing the first valid lane's bin are counted with one atomic (scores of a row
-        // crowd into few bins); the others add for themselves
+        // the lanes of a warp that share a bin are counted with one addition by the first of them
         const unsigned vm = __ballot_sync(0xffffffffu, valid);
-        if (vm) {
-            const int leader = __ffs(vm) - 1;
-            const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
-            const bool same = valid && bin == lbin;
-            const unsigned sm = __ballot_sync(0xffffffffu, same);
-            if (lane == leader) atomicAdd(&s.fine[lbin], (uint32_t)__popc(sm));
-            else if (valid && !same) atomicAdd(&s.fine[bin], 1u);
+        if (valid) {
+            const unsigned peers = __match_any_sync(vm, bin);
+            if (lane == __ffs(peers) - 1) atomicAdd(&s.fine[bin], (uint32_t)__popc(peers));
         }
     }
     __syncthreads();
