@@ -104,8 +104,8 @@ def algorithmic_bytes(cfg, kernel: str) -> float:
 # kernel inside a running step (caches as the steps before left them); see
 # profiles/kernels_llama31_8b_32k_ncu_warm.md.  Only for the workload and kernels those captures
 # cover and only while the kernels are the ones captured; anything else reports null.
-NCU_TRAFFIC = {"llama31_8b_32k": {"score_fused_tc": 74.22e6, "pool_select_sources": 0.25e6,
-                                  "similarity_tc": 0.41e6, "decay_select_gather": 1.61e6}}
+NCU_TRAFFIC = {"llama31_8b_32k": {"score_fused_tc": 73.05e6, "pool_select_sources": 0.27e6,
+                                  "similarity_tc": 0.41e6, "decay_select_gather": 1.66e6}}
 
 
 def path_bytes(cfg) -> float:
